@@ -1,0 +1,187 @@
+/*
+ * ksa.h -- C ABI of the B200 (sm_100a) Kwai Summary Attention forward library.
+ *
+ * The library computes the KSA attention operator of the paper,
+ *     O = softmax(Q K^T * scale + M_KSA) V          (student attention equation, Sec. 4.1.4)
+ * over the augmented sequence of Eq. 1 (k text tokens followed by the chunk's summary
+ * token(s), chunk after chunk), with the visibility mask M_KSA of Eq. 3 for text
+ * rows and the "own chunk only" rule of Sec. 2.2.1 for summary rows, without ever
+ * materialising the mask: a block-sparse schedule lists, per query tile, only the
+ * key/value tiles that hold at least one visible pair (the block-sparse training /
+ * prefill kernel of Sec. 2.3).
+ *
+ * Conventions
+ *   - Every function returns an int status: KSA_OK (0) or a negative KSA_ERR_* code.
+ *     Nothing throws, aborts or prints.  Invalid arguments never launch a kernel.
+ *   - "HOST" / "DEVICE" in a comment says where a pointer must live.
+ *   - The caller owns every buffer it passes (q, k, v, out, lse, workspace); the
+ *     library neither frees nor keeps them beyond the completion of the stream work
+ *     it enqueued.  A ksa_ctx owns only its cached schedule and a few small device
+ *     tables, which ksa_destroy releases.
+ *   - ksa_attn_fwd is asynchronous on the given CUDA stream and performs no host
+ *     synchronisation once the schedule for the given lengths is cached (the first
+ *     call with a new set of lengths builds and uploads it with a blocking copy).
+ *   - There is no CPU fallback: on a machine without an sm_100 device ksa_create fails.
+ *
+ * Layout of one packed batch (Eq. 1, generalised to m summaries per chunk):
+ *   sequence b has n_b text tokens, J_b = floor(n_b / k) full chunks and
+ *   L_b = n_b + J_b * m augmented rows; chunk j occupies rows j*(k+m) .. j*(k+m)+k+m-1
+ *   (k text rows, then m summary rows); a trailing partial chunk has text rows only.
+ *   Sequences are stored back to back: total_aug = sum_b L_b rows.
+ *   q, out : [total_aug, num_q_heads,  head_dim] bf16 (strides given in elements)
+ *   k, v   : [total_aug, num_kv_heads, head_dim] bf16
+ *   lse    : [num_q_heads, total_aug] fp32, natural log of sum_j exp(scale * <q, k_j>)
+ *            over the row's visible keys.
+ *   Query head h reads KV head floor(h / (num_q_heads / num_kv_heads)).
+ */
+#ifndef KSA_H
+#define KSA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------------------- */
+#define KSA_OK                 0
+#define KSA_ERR_INVALID_ARG   -1   /* null pointer, k < 1, m < 0, C < 0, bad lengths/strides/alignment */
+#define KSA_ERR_UNSUPPORTED   -2   /* head_dim not 64/128, device is not sm_100, limits exceeded      */
+#define KSA_ERR_WORKSPACE     -3   /* workspace missing or smaller than ksa_workspace_bytes            */
+#define KSA_ERR_CUDA          -4   /* a CUDA runtime/driver call failed (see ksa_last_cuda_error)      */
+#define KSA_ERR_TIMEOUT       -5   /* a bounded device-side wait gave up (see ksa_last_device_status)  */
+#define KSA_ERR_NOMEM         -6   /* host allocation failed                                           */
+
+/* ---- flags -------------------------------------------------------------------------- */
+/* Summary rows see the text of their own chunk only (strict reading of Sec. 2.2.1).
+ * Default (flag clear): summary r of a chunk also sees summaries 0..r of that chunk,
+ * itself included, as the decode procedure of Sec. 2.3.1 does. */
+#define KSA_FLAG_SUMMARY_TEXT_ONLY   0x1u
+/* Run the text rows through the plain CUDA-core cross-check kernel instead of the
+ * tensor-core kernel.  Same schedule, same packed streams; slow; for debugging. */
+#define KSA_FLAG_REFERENCE_KERNEL    0x2u
+
+typedef struct ksa_ctx ksa_ctx;    /* opaque */
+
+/* Problem statement of one forward call. */
+typedef struct ksa_params {
+    int32_t  struct_size;          /* = sizeof(ksa_params); ABI check                              */
+    int32_t  num_seqs;             /* B >= 1 packed sequences                                      */
+    const int32_t* cu_text_lens;   /* HOST, B+1 entries: prefix sums of the TEXT lengths, [0] = 0  */
+    int32_t  chunk_len;            /* k >= 1 text tokens per chunk (Eq. 1)                         */
+    int32_t  summaries_per_chunk;  /* m >= 0 (paper: 1; 0 = sliding chunk attention alone, Eq. 2)  */
+    int32_t  window_chunks;        /* C >= 0, the sliding chunk number of Eqs. 2-3                 */
+    int32_t  num_q_heads;
+    int32_t  num_kv_heads;         /* must divide num_q_heads                                      */
+    int32_t  head_dim;             /* 64 or 128; innermost, stride 1                               */
+    float    softmax_scale;        /* e.g. 1/sqrt(head_dim)                                        */
+    int64_t  q_stride_tok, q_stride_head;   /* element strides; multiples of 8                     */
+    int64_t  k_stride_tok, k_stride_head;
+    int64_t  v_stride_tok, v_stride_head;
+    int64_t  o_stride_tok, o_stride_head;
+    uint32_t flags;                /* KSA_FLAG_*                                                   */
+    uint32_t reserved;             /* must be 0                                                    */
+} ksa_params;
+
+/* One visited (query tile, key/value tile) pair of the schedule (see ksa_schedule_dump).
+ * Rows are in per-sequence STREAM coordinates: the text stream of a sequence is its
+ * text tokens 0..n-1 in order; the summary stream is its summaries in order
+ * (chunk j, slot r) -> j*m + r. */
+#define KSA_STREAM_TEXT     0
+#define KSA_STREAM_SUMMARY  1
+typedef struct ksa_tile_rec {
+    int32_t seq;
+    int32_t q_stream;              /* KSA_STREAM_TEXT (summary rows are not tiled)                 */
+    int32_t q_row0, q_rows;        /* query rows [q_row0, q_row0 + q_rows) of the text stream      */
+    int32_t kv_stream;             /* KSA_STREAM_TEXT or KSA_STREAM_SUMMARY                        */
+    int32_t kv_row0, kv_rows;      /* in-range key rows of the tile                                */
+    int32_t is_full;               /* 1: every (query, key) pair of the rectangle is visible       */
+} ksa_tile_rec;
+
+/* ---- context ------------------------------------------------------------------------ */
+/* Creates a context bound to CUDA device `cuda_device` (which becomes current on the
+ * calling thread).  Fails with KSA_ERR_UNSUPPORTED unless the device is compute
+ * capability 10.x, and with KSA_ERR_CUDA if no usable device/driver exists. */
+int ksa_create(ksa_ctx** out, int cuda_device);
+/* Releases the context's own host and device memory.  Work previously enqueued with
+ * this context must have completed.  NULL is accepted. */
+int ksa_destroy(ksa_ctx* ctx);
+
+/* ---- layout helpers (host, pure) ------------------------------------------------------ */
+/* Eq. 1: augmented length n + floor(n/k)*m of one sequence; -1 on bad arguments. */
+int64_t ksa_aug_len(int64_t n_text, int32_t k, int32_t m);
+/* Sum of ksa_aug_len over the packed batch described by p; <0 = status code. */
+int64_t ksa_total_aug_len(const ksa_params* p);
+/* Bytes of DEVICE workspace ksa_attn_fwd needs for p (packed Q/K/V streams, 256-byte
+ * aligned sub-buffers).  ctx may be NULL. */
+int ksa_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
+/* Visible (query, key) pairs of the whole batch, text and summary rows, per query
+ * head (closed form of Eq. 3); visible FLOPs = 4 * head_dim * num_q_heads * pairs. */
+int ksa_visible_pairs(const ksa_params* p, int64_t* pairs);
+
+/* ---- forward ------------------------------------------------------------------------ */
+/*
+ * KSA attention forward (Eq. 3 mask, softmax(QK^T*scale + M)V).
+ *   q, k, v   DEVICE bf16, layouts above, 16-byte aligned
+ *   out       DEVICE bf16, same shape as q (strides o_stride_*); every row is written
+ *   lse       DEVICE fp32 [num_q_heads, total_aug]; every entry is written
+ *   workspace DEVICE, >= ksa_workspace_bytes, 256-byte aligned; contents are scratch and
+ *             must not be used by other work on other streams while the call runs
+ *   cuda_stream  a cudaStream_t (NULL = legacy default stream)
+ * Steps enqueued: pack (de-interleave text Q/K/V and summary K/V into dense streams),
+ * summary-row attention, text-row attention over the scheduled tiles.
+ * Errors: KSA_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE before anything is launched;
+ * KSA_ERR_CUDA if a launch fails.  Device-side bounded waits report through
+ * ksa_last_device_status after the stream has been synchronised.
+ */
+int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v,
+                 void* out, float* lse, void* workspace, size_t workspace_bytes,
+                 const ksa_params* p, void* cuda_stream);
+
+/* Bytes of DEVICE staging ksa_attn_fwd_host needs (q, k, v, out, lse images plus the
+ * workspace of ksa_attn_fwd). */
+int ksa_host_staging_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
+/*
+ * Same operator with HOST tensors (contiguous [total_aug, H, D]; strides in p are
+ * ignored): copies q, k, v to the device staging buffer, runs ksa_attn_fwd, copies out
+ * and lse back and synchronises the stream before returning.  Pinned host memory is
+ * recommended.  staging: DEVICE, >= ksa_host_staging_bytes, 256-byte aligned.
+ */
+int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                      void* out_host, float* lse_host, void* staging, size_t staging_bytes,
+                      const ksa_params* p, void* cuda_stream);
+
+/* ---- schedule inspection ------------------------------------------------------------ */
+/*
+ * Lists every (query tile, key/value tile) pair the text-row kernel visits for p, in
+ * the order: sequence, query tile, summary tiles ascending, text tiles ascending.
+ * (Heads share the schedule.)  recs: HOST array of capacity cap (may be NULL to count);
+ * *count receives the number of records.  Returns KSA_ERR_INVALID_ARG if cap is too
+ * small (count still set).  A tile is listed iff it holds at least one visible pair.
+ */
+int ksa_schedule_dump(ksa_ctx* ctx, const ksa_params* p, ksa_tile_rec* recs, int64_t cap,
+                      int64_t* count);
+
+/* ---- diagnostics -------------------------------------------------------------------- */
+/* Reads (with a blocking copy) the device status word written by bounded waits:
+ * 0 = no wait ever gave up; otherwise a code naming the first wait that did. */
+int ksa_last_device_status(ksa_ctx* ctx, int32_t* status);
+/* Clears the device status word (blocking copy). */
+int ksa_clear_device_status(ksa_ctx* ctx);
+/* Last cudaError_t / CUresult seen by this context (0 = none). */
+int ksa_last_cuda_error(const ksa_ctx* ctx);
+/* Kernels launched by this context since creation (pack + summary + text kernels). */
+int64_t ksa_launch_count(const ksa_ctx* ctx);
+/* Optional per-kernel timing: when enabled, ksa_attn_fwd records CUDA events on the
+ * caller's stream before and after the text-row kernel (the dominant kernel).
+ * ksa_text_kernel_ms waits for the most recent pair and returns the elapsed device
+ * time in milliseconds.  Off by default (no events are recorded). */
+int ksa_enable_kernel_timing(ksa_ctx* ctx, int on);
+int ksa_text_kernel_ms(ksa_ctx* ctx, float* ms);
+const char* ksa_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KSA_H */

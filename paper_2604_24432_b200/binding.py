@@ -1,0 +1,268 @@
+"""Thin ctypes binding of ``include/ksa.h`` (same names, argument marshalling only).
+
+Every step of the forward pass runs inside the shared library's CUDA kernels; this
+module allocates nothing on the device except through torch tensors the caller (or the
+convenience wrapper ``attn_fwd``) owns.  If the shared library is missing the import of
+this module still succeeds, but every entry point raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libksa_b200.so")
+
+KSA_OK = 0
+KSA_ERR_INVALID_ARG, KSA_ERR_UNSUPPORTED, KSA_ERR_WORKSPACE = -1, -2, -3
+KSA_ERR_CUDA, KSA_ERR_TIMEOUT, KSA_ERR_NOMEM = -4, -5, -6
+KSA_FLAG_SUMMARY_TEXT_ONLY = 0x1
+KSA_FLAG_REFERENCE_KERNEL = 0x2
+KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
+
+EXPORTS = [
+    "ksa_create", "ksa_destroy", "ksa_aug_len", "ksa_total_aug_len", "ksa_workspace_bytes",
+    "ksa_visible_pairs", "ksa_attn_fwd", "ksa_host_staging_bytes", "ksa_attn_fwd_host",
+    "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
+    "ksa_last_cuda_error", "ksa_launch_count", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
+    "ksa_strerror",
+]
+
+
+class ksa_params(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_int32), ("num_seqs", ctypes.c_int32),
+        ("cu_text_lens", ctypes.c_void_p),
+        ("chunk_len", ctypes.c_int32), ("summaries_per_chunk", ctypes.c_int32),
+        ("window_chunks", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float),
+        ("q_stride_tok", ctypes.c_int64), ("q_stride_head", ctypes.c_int64),
+        ("k_stride_tok", ctypes.c_int64), ("k_stride_head", ctypes.c_int64),
+        ("v_stride_tok", ctypes.c_int64), ("v_stride_head", ctypes.c_int64),
+        ("o_stride_tok", ctypes.c_int64), ("o_stride_head", ctypes.c_int64),
+        ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+    ]
+
+
+class ksa_tile_rec(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("seq", "q_stream", "q_row0", "q_rows", "kv_stream", "kv_row0", "kv_rows", "is_full")]
+
+
+class KsaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library (built by ``paper_2604_24432_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2604_24432_b200.build` "
+            "(there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    pp = ctypes.POINTER(ksa_params)
+    L.ksa_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+    L.ksa_destroy.argtypes = [vp]
+    L.ksa_aug_len.restype = i64
+    L.ksa_aug_len.argtypes = [i64, i32, i32]
+    L.ksa_total_aug_len.restype = i64
+    L.ksa_total_aug_len.argtypes = [pp]
+    L.ksa_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
+    L.ksa_visible_pairs.argtypes = [pp, ctypes.POINTER(i64)]
+    L.ksa_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
+    L.ksa_host_staging_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
+    L.ksa_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
+    L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
+    L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.ksa_clear_device_status.argtypes = [vp]
+    L.ksa_last_cuda_error.argtypes = [vp]
+    L.ksa_launch_count.restype = i64
+    L.ksa_launch_count.argtypes = [vp]
+    L.ksa_enable_kernel_timing.argtypes = [vp, ctypes.c_int]
+    L.ksa_text_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    L.ksa_strerror.restype = ctypes.c_char_p
+    L.ksa_strerror.argtypes = [ctypes.c_int]
+    _lib = L
+    return L
+
+
+def strerror(status: int) -> str:
+    return lib().ksa_strerror(status).decode()
+
+
+def _check(status: int, where: str):
+    if status != KSA_OK:
+        raise KsaError(status, where)
+
+
+@dataclass
+class Problem:
+    """Python-side holder of a ``ksa_params`` plus the host array it points to."""
+    text_lens: Sequence[int]
+    k: int
+    m: int
+    C: int
+    Hq: int
+    Hkv: int
+    D: int
+    scale: float
+    flags: int = 0
+
+    def params(self, q=None, k=None, v=None, o=None) -> ksa_params:
+        cu = np.concatenate([[0], np.cumsum(np.asarray(self.text_lens, dtype=np.int64))]).astype(np.int32)
+        self._cu = cu  # keep alive
+        p = ksa_params()
+        p.struct_size = ctypes.sizeof(ksa_params)
+        p.num_seqs = len(self.text_lens)
+        p.cu_text_lens = cu.ctypes.data
+        p.chunk_len, p.summaries_per_chunk, p.window_chunks = self.k, self.m, self.C
+        p.num_q_heads, p.num_kv_heads, p.head_dim = self.Hq, self.Hkv, self.D
+        p.softmax_scale = self.scale
+        p.flags = self.flags
+        p.reserved = 0
+
+        def strides(t, H):
+            if t is None:
+                return H * self.D, self.D
+            assert t.stride(2) == 1, "head_dim must be contiguous"
+            return t.stride(0), t.stride(1)
+
+        p.q_stride_tok, p.q_stride_head = strides(q, self.Hq)
+        p.k_stride_tok, p.k_stride_head = strides(k, self.Hkv)
+        p.v_stride_tok, p.v_stride_head = strides(v, self.Hkv)
+        p.o_stride_tok, p.o_stride_head = strides(o, self.Hq)
+        return p
+
+
+def aug_len(n_text: int, k: int, m: int) -> int:
+    return int(lib().ksa_aug_len(n_text, k, m))
+
+
+def total_aug_len(prob: Problem) -> int:
+    p = prob.params()
+    r = int(lib().ksa_total_aug_len(ctypes.byref(p)))
+    if r < 0:
+        raise KsaError(r, "ksa_total_aug_len")
+    return r
+
+
+def workspace_bytes(prob: Problem) -> int:
+    p = prob.params()
+    n = ctypes.c_size_t()
+    _check(lib().ksa_workspace_bytes(None, ctypes.byref(p), ctypes.byref(n)), "ksa_workspace_bytes")
+    return int(n.value)
+
+
+def host_staging_bytes(prob: Problem) -> int:
+    p = prob.params()
+    n = ctypes.c_size_t()
+    _check(lib().ksa_host_staging_bytes(None, ctypes.byref(p), ctypes.byref(n)), "ksa_host_staging_bytes")
+    return int(n.value)
+
+
+def visible_pairs(prob: Problem) -> int:
+    p = prob.params()
+    n = ctypes.c_int64()
+    _check(lib().ksa_visible_pairs(ctypes.byref(p), ctypes.byref(n)), "ksa_visible_pairs")
+    return int(n.value)
+
+
+def schedule_dump(prob: Problem, ctx: Optional["Context"] = None) -> np.ndarray:
+    """Structured numpy array of the visited (query tile, kv tile) records."""
+    p = prob.params()
+    cnt = ctypes.c_int64()
+    h = ctx.handle if ctx is not None else None
+    _check(lib().ksa_schedule_dump(h, ctypes.byref(p), None, 0, ctypes.byref(cnt)), "ksa_schedule_dump")
+    arr = (ksa_tile_rec * max(1, cnt.value))()
+    _check(lib().ksa_schedule_dump(h, ctypes.byref(p), arr, cnt.value, ctypes.byref(cnt)), "ksa_schedule_dump")
+    dt = np.dtype([(n, np.int32) for n, _ in ksa_tile_rec._fields_])
+    return np.frombuffer(arr, dtype=dt, count=cnt.value).copy()
+
+
+class Context:
+    """Owns a ``ksa_ctx``."""
+
+    def __init__(self, device: int = 0):
+        h = ctypes.c_void_p()
+        _check(lib().ksa_create(ctypes.byref(h), device), "ksa_create")
+        self.handle = h
+        self.device = device
+
+    def close(self):
+        if self.handle:
+            lib().ksa_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def attn_fwd(self, prob: Problem, q, k, v, out, lse, workspace, stream: Optional[int] = None):
+        """ksa_attn_fwd on torch CUDA tensors (q, k, v, out bf16; lse fp32; workspace uint8)."""
+        import torch
+        p = prob.params(q, k, v, out)
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        _check(lib().ksa_attn_fwd(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                  lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                  ctypes.byref(p), stream), "ksa_attn_fwd")
+
+    def attn_fwd_host(self, prob: Problem, q, k, v, out, lse, staging, stream: Optional[int] = None):
+        """ksa_attn_fwd_host: q, k, v, out, lse are contiguous HOST tensors (pinned recommended)."""
+        import torch
+        p = prob.params()
+        if stream is None:
+            stream = torch.cuda.current_stream(staging.device).cuda_stream
+        _check(lib().ksa_attn_fwd_host(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                       lse.data_ptr(), staging.data_ptr(), staging.numel() * staging.element_size(),
+                                       ctypes.byref(p), stream), "ksa_attn_fwd_host")
+
+    def device_status(self) -> int:
+        s = ctypes.c_int32()
+        _check(lib().ksa_last_device_status(self.handle, ctypes.byref(s)), "ksa_last_device_status")
+        return int(s.value)
+
+    def clear_device_status(self):
+        _check(lib().ksa_clear_device_status(self.handle), "ksa_clear_device_status")
+
+    def last_cuda_error(self) -> int:
+        return int(lib().ksa_last_cuda_error(self.handle))
+
+    def launch_count(self) -> int:
+        return int(lib().ksa_launch_count(self.handle))
+
+    def enable_kernel_timing(self, on: bool = True):
+        _check(lib().ksa_enable_kernel_timing(self.handle, int(on)), "ksa_enable_kernel_timing")
+
+    def text_kernel_ms(self) -> float:
+        ms = ctypes.c_float()
+        _check(lib().ksa_text_kernel_ms(self.handle, ctypes.byref(ms)), "ksa_text_kernel_ms")
+        return float(ms.value)
+
+
+def attn_fwd(ctx: Context, prob: Problem, q, k, v):
+    """Convenience wrapper: allocates out, lse and the workspace with torch and calls
+    ``ksa_attn_fwd`` on the current stream.  Returns (out, lse)."""
+    import torch
+    total = q.shape[0]
+    out = torch.empty((total, prob.Hq, prob.D), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((prob.Hq, total), dtype=torch.float32, device=q.device)
+    ws = torch.empty(workspace_bytes(prob), dtype=torch.uint8, device=q.device)
+    ctx.attn_fwd(prob, q, k, v, out, lse, ws)
+    return out, lse

@@ -1,0 +1,608 @@
+// C ABI of the KSA forward library: argument validation, sequence layout (Eq. 1), the
+// block-sparse tile schedule (Eq. 3 at tile granularity) and the kernel launches.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/ksa.h"
+#include "ksa_launch.h"
+
+using namespace ksa;
+
+static_assert(sizeof(ksa_params) == 120, "ksa_params ABI");
+static_assert(sizeof(ksa_tile_rec) == 32, "ksa_tile_rec ABI");
+
+// ---------------------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct HostSchedule {
+    std::vector<int32_t> key;         // lengths and parameters this schedule was built for
+    std::vector<SeqInfo> seqs;
+    std::vector<WorkItem> work;       // sorted, longest first
+    int64_t total_aug = 0, text_rows = 0, summ_rows = 0;
+    int32_t max_text_pad = 0, max_summ_pad = 0, max_n_summ = 0;
+};
+
+struct ksa_ctx {
+    int device = -1;
+    int num_sms = 0;
+    int last_cuda_error = 0;
+    int64_t launches = 0;
+    EncodeTiledFn encode = nullptr;
+    HostSchedule sched;               // cached schedule (one entry)
+    SeqInfo* d_seqs = nullptr;  size_t d_seqs_cap = 0;
+    WorkItem* d_work = nullptr; size_t d_work_cap = 0;
+    int32_t* d_status = nullptr;
+    bool timing = false;
+    bool timing_valid = false;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    bool tc_ready = false;
+};
+
+static int cuda_fail(ksa_ctx* ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return KSA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// validation and layout
+// ---------------------------------------------------------------------------------------
+static int validate(const ksa_params* p)
+{
+    if (!p || p->struct_size != (int32_t)sizeof(ksa_params)) return KSA_ERR_INVALID_ARG;
+    if (p->num_seqs < 1 || !p->cu_text_lens) return KSA_ERR_INVALID_ARG;
+    if (p->chunk_len < 1 || p->summaries_per_chunk < 0 || p->window_chunks < 0) return KSA_ERR_INVALID_ARG;
+    if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
+        return KSA_ERR_INVALID_ARG;
+    if (p->reserved != 0) return KSA_ERR_INVALID_ARG;
+    if (p->flags & ~(KSA_FLAG_SUMMARY_TEXT_ONLY | KSA_FLAG_REFERENCE_KERNEL)) return KSA_ERR_INVALID_ARG;
+    if (!(p->softmax_scale > 0.f) || !std::isfinite(p->softmax_scale)) return KSA_ERR_INVALID_ARG;
+    if (p->cu_text_lens[0] != 0) return KSA_ERR_INVALID_ARG;
+    for (int b = 0; b < p->num_seqs; ++b)
+        if (p->cu_text_lens[b + 1] <= p->cu_text_lens[b]) return KSA_ERR_INVALID_ARG;  // empty or non-monotone
+    if (p->head_dim != 64 && p->head_dim != 128) return KSA_ERR_UNSUPPORTED;
+    if (p->num_q_heads > 1024 || p->chunk_len > (1 << 20) || p->summaries_per_chunk > (1 << 20))
+        return KSA_ERR_UNSUPPORTED;
+    // padded stream rows must fit comfortably in int32
+    int64_t n_total = p->cu_text_lens[p->num_seqs];
+    if (n_total + (int64_t)p->num_seqs * kTileM > (1ll << 30)) return KSA_ERR_UNSUPPORTED;
+    if (n_total / p->chunk_len * (int64_t)p->summaries_per_chunk + (int64_t)p->num_seqs * kTileN > (1ll << 30))
+        return KSA_ERR_UNSUPPORTED;
+    return KSA_OK;
+}
+
+static int validate_strides(const ksa_params* p)
+{
+    const int64_t st[8] = {p->q_stride_tok, p->q_stride_head, p->k_stride_tok, p->k_stride_head,
+                           p->v_stride_tok, p->v_stride_head, p->o_stride_tok, p->o_stride_head};
+    for (int i = 0; i < 8; ++i)
+        if (st[i] < p->head_dim || (st[i] % 8) != 0) return KSA_ERR_INVALID_ARG;
+    return KSA_OK;
+}
+
+static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+static void build_layout(const ksa_params* p, HostSchedule& hs)
+{
+    const int k = p->chunk_len, m = p->summaries_per_chunk;
+    hs.seqs.resize(p->num_seqs);
+    int64_t aug = 0, trow = 0, srow = 0;
+    hs.max_text_pad = hs.max_summ_pad = hs.max_n_summ = 0;
+    for (int b = 0; b < p->num_seqs; ++b) {
+        SeqInfo& s = hs.seqs[b];
+        std::memset(&s, 0, sizeof s);
+        s.n_text = p->cu_text_lens[b + 1] - p->cu_text_lens[b];
+        s.n_chunks = s.n_text / k;                        // only full chunks carry summaries
+        s.n_summ = s.n_chunks * m;
+        s.aug_off = aug;
+        s.text_off = (int32_t)trow;
+        s.summ_off = (int32_t)srow;
+        s.text_pad = (int32_t)round_up(s.n_text, kTileM);
+        s.summ_pad = (int32_t)round_up(s.n_summ, kTileN);
+        aug += (int64_t)s.n_text + s.n_summ;              // Eq. 1: L = n + floor(n/k) m
+        trow += s.text_pad;
+        srow += s.summ_pad;
+        hs.max_text_pad = std::max(hs.max_text_pad, s.text_pad);
+        hs.max_summ_pad = std::max(hs.max_summ_pad, s.summ_pad);
+        hs.max_n_summ = std::max(hs.max_n_summ, s.n_summ);
+    }
+    hs.total_aug = aug;
+    hs.text_rows = trow;
+    hs.summ_rows = std::max<int64_t>(srow, kTileN);       // keep the tensor maps non-empty
+}
+
+// ---------------------------------------------------------------------------------------
+// Eq. 3 at tile granularity.  For text row i of a sequence (chunk c = i / k):
+//   first visible text token   lo(i)  = max(0, c - C) * k
+//   visible summary rows       [0, cnt(i)),  cnt(i) = max(0, c - C) * m
+// Both are non-decreasing in i, which makes the visited tiles of a query tile two
+// contiguous ranges and the unmasked tiles contiguous sub-ranges.
+// ---------------------------------------------------------------------------------------
+struct Eq3 {
+    int k, m, C;
+    int64_t lo(int64_t i) const { return std::max<int64_t>(0, i / k - C) * k; }
+    int64_t cnt(int64_t i) const { return std::max<int64_t>(0, i / k - C) * m; }
+};
+struct TileClass { bool any, full; };
+
+// query rows [i0, i1], text key rows [a0, a1] (all in range)
+static TileClass classify_text(const Eq3& e, int64_t i0, int64_t i1, int64_t a0, int64_t a1)
+{
+    TileClass t;
+    const int64_t ifirst = std::max(i0, a0);              // first row that can reach the tile causally
+    t.any = (ifirst <= i1) && (e.lo(ifirst) <= a1);
+    t.full = (e.lo(i1) <= a0) && (i0 >= a1);
+    return t;
+}
+// query rows [i0, i1], summary stream rows [u0, u1]
+static TileClass classify_summ(const Eq3& e, int64_t i0, int64_t i1, int64_t u0, int64_t u1)
+{
+    TileClass t;
+    t.any = e.cnt(i1) > u0;
+    t.full = e.cnt(i0) > u1;
+    return t;
+}
+
+struct BaseItem {   // schedule of one (sequence, query tile); heads share it
+    int32_t seq, q_tile, ns_tiles, ns_nomask, band_lo, band_hi, nm_lo, nm_hi;
+};
+
+static BaseItem schedule_q_tile(const Eq3& e, const SeqInfo& s, int seq, int qt)
+{
+    BaseItem it{};
+    it.seq = seq;
+    it.q_tile = qt;
+    const int64_t i0 = (int64_t)qt * kTileM;
+    const int64_t i1 = std::min<int64_t>(s.n_text, i0 + kTileM) - 1;
+    // summary stream: tiles [0, ceil(cnt(i1) / kTileN))
+    const int64_t cmax = std::min<int64_t>(e.cnt(i1), s.n_summ);
+    it.ns_tiles = (int32_t)((cmax + kTileN - 1) / kTileN);
+    it.ns_nomask = 0;
+    for (int ut = 0; ut < it.ns_tiles; ++ut) {
+        const int64_t u0 = (int64_t)ut * kTileN, u1 = std::min<int64_t>(s.n_summ, u0 + kTileN) - 1;
+        const TileClass tc = classify_summ(e, i0, i1, u0, u1);
+        if (tc.full && (u1 - u0 + 1) == kTileN && it.ns_nomask == ut) it.ns_nomask = ut + 1;
+    }
+    // text stream: tiles [lo(i0) / kTileN, qt]
+    it.band_lo = (int32_t)(e.lo(i0) / kTileN);
+    it.band_hi = qt;
+    it.nm_lo = it.nm_hi = it.band_lo;
+    bool open = false, closed = false;
+    for (int bt = it.band_lo; bt <= it.band_hi; ++bt) {
+        const int64_t a0 = (int64_t)bt * kTileN, a1 = std::min<int64_t>(s.n_text, a0 + kTileN) - 1;
+        const TileClass tc = classify_text(e, i0, i1, a0, a1);
+        const bool nomask = tc.full && (a1 - a0 + 1) == kTileN;
+        if (nomask && !open && !closed) { open = true; it.nm_lo = bt; it.nm_hi = bt + 1; }
+        else if (nomask && open) it.nm_hi = bt + 1;
+        else if (!nomask && open) { open = false; closed = true; }
+    }
+    return it;
+}
+
+static void build_schedule(const ksa_params* p, HostSchedule& hs)
+{
+    const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const int heads_per_item = (G % 2 == 0) ? 2 : 1;
+    std::vector<BaseItem> base;
+    for (int b = 0; b < p->num_seqs; ++b) {
+        const int n_qt = hs.seqs[b].text_pad / kTileM;
+        for (int qt = 0; qt < n_qt; ++qt) base.push_back(schedule_q_tile(e, hs.seqs[b], b, qt));
+    }
+    // longest first; ties keep (sequence, tile) order so that neighbours share K/V tiles in L2
+    std::stable_sort(base.begin(), base.end(), [](const BaseItem& x, const BaseItem& y) {
+        return (x.ns_tiles + x.band_hi - x.band_lo) > (y.ns_tiles + y.band_hi - y.band_lo);
+    });
+    hs.work.clear();
+    hs.work.reserve(base.size() * (p->num_q_heads / heads_per_item));
+    for (const BaseItem& bi : base)
+        for (int h = 0; h < p->num_q_heads; h += heads_per_item) {
+            WorkItem w{};
+            w.seq = bi.seq; w.q_tile = bi.q_tile; w.head0 = h; w.n_heads = heads_per_item;
+            w.ns_tiles = bi.ns_tiles; w.ns_nomask = bi.ns_nomask;
+            w.band_lo = bi.band_lo; w.band_hi = bi.band_hi;
+            w.band_nomask_lo = bi.nm_lo; w.band_nomask_hi = bi.nm_hi;
+            hs.work.push_back(w);
+        }
+}
+
+static std::vector<int32_t> schedule_key(const ksa_params* p)
+{
+    std::vector<int32_t> key;
+    key.reserve(p->num_seqs + 8);
+    key.push_back(p->num_seqs);
+    for (int b = 0; b <= p->num_seqs; ++b) key.push_back(p->cu_text_lens[b]);
+    key.push_back(p->chunk_len); key.push_back(p->summaries_per_chunk); key.push_back(p->window_chunks);
+    key.push_back(p->num_q_heads); key.push_back(p->num_kv_heads); key.push_back(p->head_dim);
+    return key;
+}
+
+struct WorkspaceLayout { size_t qt, kt, vt, ks, vs, total; };
+static WorkspaceLayout workspace_layout(const ksa_params* p, const HostSchedule& hs)
+{
+    WorkspaceLayout w{};
+    const size_t D2 = (size_t)p->head_dim * 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
+    w.qt = take((size_t)p->num_q_heads * hs.text_rows * D2);
+    w.kt = take((size_t)p->num_kv_heads * hs.text_rows * D2);
+    w.vt = take((size_t)p->num_kv_heads * hs.text_rows * D2);
+    w.ks = take((size_t)p->num_kv_heads * hs.summ_rows * D2);
+    w.vs = take((size_t)p->num_kv_heads * hs.summ_rows * D2);
+    w.total = off;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------
+// exported: helpers
+// ---------------------------------------------------------------------------------------
+extern "C" __attribute__((visibility("default"))) int64_t ksa_aug_len(int64_t n_text, int32_t k, int32_t m)
+{
+    if (n_text < 0 || k < 1 || m < 0) return -1;
+    return n_text + (n_text / k) * (int64_t)m;
+}
+
+extern "C" __attribute__((visibility("default"))) int64_t ksa_total_aug_len(const ksa_params* p)
+{
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    int64_t t = 0;
+    for (int b = 0; b < p->num_seqs; ++b)
+        t += ksa_aug_len(p->cu_text_lens[b + 1] - p->cu_text_lens[b], p->chunk_len, p->summaries_per_chunk);
+    return t;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_workspace_bytes(const ksa_ctx*, const ksa_params* p, size_t* bytes)
+{
+    if (!bytes) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    HostSchedule hs;
+    build_layout(p, hs);
+    *bytes = workspace_layout(p, hs).total;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_visible_pairs(const ksa_params* p, int64_t* pairs)
+{
+    if (!pairs) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
+    const int64_t k = p->chunk_len, m = p->summaries_per_chunk;
+    int64_t total = 0;
+    for (int b = 0; b < p->num_seqs; ++b) {
+        const int64_t n = p->cu_text_lens[b + 1] - p->cu_text_lens[b];
+        for (int64_t c = 0; c * k < n; ++c) {             // rows of chunk c: i = ck .. min(n, ck+k)-1
+            const int64_t rows = std::min(n, c * k + k) - c * k;
+            const int64_t i0 = c * k;
+            // sum over rows of (i - lo + 1) + cnt
+            total += rows * (i0 - e.lo(i0) + 1 + e.cnt(i0)) + rows * (rows - 1) / 2;
+        }
+        const int64_t J = n / k;
+        for (int64_t r = 0; r < m; ++r)
+            total += J * (k + ((p->flags & KSA_FLAG_SUMMARY_TEXT_ONLY) ? 0 : r + 1));
+    }
+    *pairs = total;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) const char* ksa_strerror(int status)
+{
+    switch (status) {
+        case KSA_OK: return "ok";
+        case KSA_ERR_INVALID_ARG: return "invalid argument";
+        case KSA_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case KSA_ERR_WORKSPACE: return "workspace missing or too small";
+        case KSA_ERR_CUDA: return "CUDA call failed";
+        case KSA_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case KSA_ERR_NOMEM: return "out of host memory";
+        default: return "unknown status";
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// exported: context
+// ---------------------------------------------------------------------------------------
+extern "C" __attribute__((visibility("default"))) int ksa_create(ksa_ctx** out, int cuda_device)
+{
+    if (!out) return KSA_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return KSA_ERR_CUDA;
+    if (cuda_device < 0 || cuda_device >= count) return KSA_ERR_INVALID_ARG;
+    if ((e = cudaSetDevice(cuda_device)) != cudaSuccess) return KSA_ERR_CUDA;
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, cuda_device)) != cudaSuccess) return KSA_ERR_CUDA;
+    if (prop.major != 10) return KSA_ERR_UNSUPPORTED;     // kernels are built for sm_100a only
+    ksa_ctx* ctx = new (std::nothrow) ksa_ctx();
+    if (!ctx) return KSA_ERR_NOMEM;
+    ctx->device = cuda_device;
+    ctx->num_sms = prop.multiProcessorCount;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) { delete ctx; return KSA_ERR_CUDA; }
+    ctx->encode = (EncodeTiledFn)fn;
+    if ((e = cudaMalloc(&ctx->d_status, sizeof(int32_t))) != cudaSuccess) { delete ctx; return KSA_ERR_CUDA; }
+    if ((e = cudaMemset(ctx->d_status, 0, sizeof(int32_t))) != cudaSuccess) { cudaFree(ctx->d_status); delete ctx; return KSA_ERR_CUDA; }
+    cudaEventCreate(&ctx->ev0);
+    cudaEventCreate(&ctx->ev1);
+    *out = ctx;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_destroy(ksa_ctx* ctx)
+{
+    if (!ctx) return KSA_OK;
+    cudaSetDevice(ctx->device);
+    if (ctx->d_seqs) cudaFree(ctx->d_seqs);
+    if (ctx->d_work) cudaFree(ctx->d_work);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+    if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    delete ctx;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_last_device_status(ksa_ctx* ctx, int32_t* status)
+{
+    if (!ctx || !status) return KSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaMemcpy(status, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? KSA_OK : cuda_fail(ctx, e);
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_clear_device_status(ksa_ctx* ctx)
+{
+    if (!ctx) return KSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
+    return e == cudaSuccess ? KSA_OK : cuda_fail(ctx, e);
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_last_cuda_error(const ksa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+extern "C" __attribute__((visibility("default"))) int64_t ksa_launch_count(const ksa_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" __attribute__((visibility("default"))) int ksa_enable_kernel_timing(ksa_ctx* ctx, int on)
+{
+    if (!ctx) return KSA_ERR_INVALID_ARG;
+    ctx->timing = on != 0;
+    ctx->timing_valid = false;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_text_kernel_ms(ksa_ctx* ctx, float* ms)
+{
+    if (!ctx || !ms || !ctx->timing_valid) return KSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaEventSynchronize(ctx->ev1);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = cudaEventElapsedTime(ms, ctx->ev0, ctx->ev1);
+    return e == cudaSuccess ? KSA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------
+// schedule cache
+// ---------------------------------------------------------------------------------------
+static int ensure_schedule(ksa_ctx* ctx, const ksa_params* p, bool upload)
+{
+    std::vector<int32_t> key = schedule_key(p);
+    if (ctx->sched.key != key) {
+        HostSchedule hs;
+        try {
+            build_layout(p, hs);
+            build_schedule(p, hs);
+        } catch (const std::bad_alloc&) { return KSA_ERR_NOMEM; }
+        hs.key = key;
+        ctx->sched = std::move(hs);
+        // the device copies belong to the old schedule (cudaFree waits for work in flight)
+        if (ctx->d_seqs) { cudaFree(ctx->d_seqs); ctx->d_seqs = nullptr; ctx->d_seqs_cap = 0; }
+        if (ctx->d_work) { cudaFree(ctx->d_work); ctx->d_work = nullptr; ctx->d_work_cap = 0; }
+    }
+    if (upload && !ctx->d_seqs) {
+        const HostSchedule& hs = ctx->sched;
+        cudaError_t e;
+        const size_t sb = hs.seqs.size() * sizeof(SeqInfo), wb = std::max<size_t>(1, hs.work.size()) * sizeof(WorkItem);
+        if ((e = cudaMalloc(&ctx->d_seqs, sb)) != cudaSuccess) { ctx->d_seqs = nullptr; return cuda_fail(ctx, e); }
+        if ((e = cudaMalloc(&ctx->d_work, wb)) != cudaSuccess) {
+            cudaFree(ctx->d_seqs); ctx->d_seqs = nullptr; ctx->d_work = nullptr; return cuda_fail(ctx, e);
+        }
+        e = cudaMemcpy(ctx->d_seqs, hs.seqs.data(), sb, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && !hs.work.empty())
+            e = cudaMemcpy(ctx->d_work, hs.work.data(), hs.work.size() * sizeof(WorkItem), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            cudaFree(ctx->d_seqs); cudaFree(ctx->d_work); ctx->d_seqs = nullptr; ctx->d_work = nullptr;
+            return cuda_fail(ctx, e);
+        }
+        ctx->d_seqs_cap = sb; ctx->d_work_cap = wb;
+    }
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_schedule_dump(ksa_ctx* ctx, const ksa_params* p, ksa_tile_rec* recs, int64_t cap,
+                                 int64_t* count)
+{
+    if (!count) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    HostSchedule local;
+    build_layout(p, local);
+    const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
+    int64_t n = 0;
+    bool overflow = false;
+    auto emit = [&](const ksa_tile_rec& r) {
+        if (recs && n < cap) recs[n] = r; else if (recs) overflow = true;
+        ++n;
+    };
+    (void)ctx;
+    for (int b = 0; b < p->num_seqs; ++b) {
+        const SeqInfo& s = local.seqs[b];
+        for (int qt = 0; qt < s.text_pad / kTileM; ++qt) {
+            const BaseItem it = schedule_q_tile(e, s, b, qt);
+            const int64_t i0 = (int64_t)qt * kTileM, i1 = std::min<int64_t>(s.n_text, i0 + kTileM) - 1;
+            ksa_tile_rec r{};
+            r.seq = b; r.q_stream = KSA_STREAM_TEXT; r.q_row0 = (int32_t)i0; r.q_rows = (int32_t)(i1 - i0 + 1);
+            for (int ut = 0; ut < it.ns_tiles; ++ut) {
+                const int64_t u0 = (int64_t)ut * kTileN, u1 = std::min<int64_t>(s.n_summ, u0 + kTileN) - 1;
+                r.kv_stream = KSA_STREAM_SUMMARY; r.kv_row0 = (int32_t)u0; r.kv_rows = (int32_t)(u1 - u0 + 1);
+                r.is_full = classify_summ(e, i0, i1, u0, u1).full ? 1 : 0;
+                emit(r);
+            }
+            for (int bt = it.band_lo; bt <= it.band_hi; ++bt) {
+                const int64_t a0 = (int64_t)bt * kTileN, a1 = std::min<int64_t>(s.n_text, a0 + kTileN) - 1;
+                r.kv_stream = KSA_STREAM_TEXT; r.kv_row0 = (int32_t)a0; r.kv_rows = (int32_t)(a1 - a0 + 1);
+                r.is_full = classify_text(e, i0, i1, a0, a1).full ? 1 : 0;
+                emit(r);
+            }
+        }
+    }
+    *count = n;
+    return overflow ? KSA_ERR_INVALID_ARG : KSA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// forward
+// ---------------------------------------------------------------------------------------
+static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return KSA_ERR_CUDA; }
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, void* out, float* lse,
+                            void* workspace, size_t workspace_bytes, const ksa_params* p, void* cuda_stream)
+{
+    if (!ctx || !q || !k || !v || !out || !lse) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = validate_strides(p)) != KSA_OK) return rc;
+    const uintptr_t ptrs[5] = {(uintptr_t)q, (uintptr_t)k, (uintptr_t)v, (uintptr_t)out, (uintptr_t)lse};
+    for (int i = 0; i < 5; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
+    if ((rc = ensure_schedule(ctx, p, true)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    const WorkspaceLayout wl = workspace_layout(p, hs);
+    if (!workspace || workspace_bytes < wl.total || ((uintptr_t)workspace & 255)) return KSA_ERR_WORKSPACE;
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* ws = (char*)workspace;
+    KernelArgs a{};
+    a.seqs = ctx->d_seqs; a.work = ctx->d_work;
+    a.num_seqs = p->num_seqs; a.num_work = (int32_t)hs.work.size();
+    a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.C = p->window_chunks;
+    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.flags = p->flags;
+    a.scale = p->softmax_scale;
+    a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+    a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
+    a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
+    a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v;
+    a.out = (uint16_t*)out; a.lse = lse;
+    a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;
+    a.v_st = p->v_stride_tok; a.v_sh = p->v_stride_head; a.o_st = p->o_stride_tok; a.o_sh = p->o_stride_head;
+    a.qt = (uint16_t*)(ws + wl.qt); a.kt = (uint16_t*)(ws + wl.kt); a.vt = (uint16_t*)(ws + wl.vt);
+    a.ks = (uint16_t*)(ws + wl.ks); a.vs = (uint16_t*)(ws + wl.vs);
+    a.status = ctx->d_status;
+
+    cudaError_t e;
+    if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    if (a.m > 0 && a.max_n_summ > 0) {
+        if ((e = launch_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
+    if (ctx->timing) cudaEventRecord(ctx->ev0, stream);
+    if (p->flags & KSA_FLAG_REFERENCE_KERNEL) {
+        if ((e = launch_text_ref(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    } else {
+        if (!ctx->tc_ready) {
+            if ((e = setup_text_tc()) != cudaSuccess) return cuda_fail(ctx, e);
+            ctx->tc_ready = true;
+        }
+        TextMaps maps;
+        if ((rc = encode_stream_map(ctx, &maps.qt, a.qt, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &maps.kt, a.kt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &maps.vt, a.vt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &maps.ks, a.ks, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &maps.vs, a.vs, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((e = launch_text_tc(a, maps, ctx->num_sms, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    ctx->launches += 1;
+    if (ctx->timing) { cudaEventRecord(ctx->ev1, stream); ctx->timing_valid = true; }
+    return KSA_OK;
+}
+
+struct StagingLayout { size_t q, k, v, out, lse, ws, ws_bytes, total; };
+static int staging_layout(const ksa_params* p, StagingLayout& s)
+{
+    HostSchedule hs;
+    build_layout(p, hs);
+    const size_t D2 = (size_t)p->head_dim * 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
+    s.q = take((size_t)hs.total_aug * p->num_q_heads * D2);
+    s.k = take((size_t)hs.total_aug * p->num_kv_heads * D2);
+    s.v = take((size_t)hs.total_aug * p->num_kv_heads * D2);
+    s.out = take((size_t)hs.total_aug * p->num_q_heads * D2);
+    s.lse = take((size_t)hs.total_aug * p->num_q_heads * 4);
+    s.ws_bytes = workspace_layout(p, hs).total;
+    s.ws = take(s.ws_bytes);
+    s.total = off;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_host_staging_bytes(const ksa_ctx*, const ksa_params* p, size_t* bytes)
+{
+    if (!bytes) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    StagingLayout s;
+    staging_layout(p, s);
+    *bytes = s.total;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                                 void* out_host, float* lse_host, void* staging, size_t staging_bytes,
+                                 const ksa_params* p, void* cuda_stream)
+{
+    if (!ctx || !q_host || !k_host || !v_host || !out_host || !lse_host) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    StagingLayout s;
+    staging_layout(p, s);
+    if (!staging || staging_bytes < s.total || ((uintptr_t)staging & 255)) return KSA_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* d = (char*)staging;
+    const size_t D2 = (size_t)p->head_dim * 2;
+    const int64_t total_aug = ksa_total_aug_len(p);
+    const size_t qb = (size_t)total_aug * p->num_q_heads * D2, kb = (size_t)total_aug * p->num_kv_heads * D2;
+    const size_t lb = (size_t)total_aug * p->num_q_heads * 4;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d + s.q, q_host, qb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(d + s.k, k_host, kb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(d + s.v, v_host, kb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    ksa_params pc = *p;   // contiguous device images
+    pc.q_stride_tok = pc.o_stride_tok = (int64_t)p->num_q_heads * p->head_dim;
+    pc.k_stride_tok = pc.v_stride_tok = (int64_t)p->num_kv_heads * p->head_dim;
+    pc.q_stride_head = pc.k_stride_head = pc.v_stride_head = pc.o_stride_head = p->head_dim;
+    rc = ksa_attn_fwd(ctx, d + s.q, d + s.k, d + s.v, d + s.out, (float*)(d + s.lse), d + s.ws, s.ws_bytes, &pc, stream);
+    if (rc != KSA_OK) return rc;
+    if ((e = cudaMemcpyAsync(out_host, d + s.out, qb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(lse_host, d + s.lse, lb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    return KSA_OK;
+}

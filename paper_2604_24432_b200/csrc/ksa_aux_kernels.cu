@@ -1,0 +1,237 @@
+// Pack (de-interleave) kernel, summary-row kernel and the CUDA-core cross-check
+// kernel for text rows.  All three are bandwidth- or latency-bound helpers around the
+// tensor-core text kernel.
+#include <cuda_bf16.h>
+
+#include "ksa_launch.h"
+
+namespace ksa {
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
+{
+    __nv_bfloat16 h = __float2bfloat16_rn(f);
+    return *reinterpret_cast<uint16_t*>(&h);
+}
+
+// ---------------------------------------------------------------------------------------
+// Pack.  grid = (blocks, num_seqs, 2): z = 0 packs the text stream (Q, K, V rows of text
+// tokens), z = 1 the summary stream (K, V rows of summary tokens).  One thread moves one
+// 16-byte vector.  Text token i of a sequence sits at augmented row (i/k)*(k+m) + i%k,
+// summary (j, r) at j*(k+m) + k + r (Eq. 1).
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) ksa_pack_kernel(KernelArgs a)
+{
+    const SeqInfo sq = a.seqs[blockIdx.y];
+    const bool text = (blockIdx.z == 0);
+    const int vecs = a.D / 8;
+    const int slots = text ? (a.Hq + 2 * a.Hkv) : (2 * a.Hkv);
+    const int pad_rows = text ? sq.text_pad : sq.summ_pad;
+    const int live_rows = text ? sq.n_text : sq.n_summ;
+    const int64_t per_row = (int64_t)slots * vecs;
+    const int64_t total = (int64_t)pad_rows * per_row;
+    const int s = a.k + a.m;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int row = (int)(idx / per_row);
+        const int rem = (int)(idx - (int64_t)row * per_row);
+        const int slot = rem / vecs;
+        const int vec = rem - slot * vecs;
+        int64_t aug = 0;
+        if (row < live_rows) {
+            if (text) aug = sq.aug_off + (int64_t)(row / a.k) * s + (row % a.k);
+            else      aug = sq.aug_off + (int64_t)(row / a.m) * s + a.k + (row % a.m);
+        }
+        const uint16_t* src;
+        uint16_t* dst;
+        if (text) {
+            const int64_t drow = (int64_t)sq.text_off + row;
+            if (slot < a.Hq) {
+                src = a.q + aug * a.q_st + (int64_t)slot * a.q_sh;
+                dst = a.qt + ((int64_t)slot * a.text_rows + drow) * a.D;
+            } else if (slot < a.Hq + a.Hkv) {
+                const int h = slot - a.Hq;
+                src = a.kx + aug * a.k_st + (int64_t)h * a.k_sh;
+                dst = a.kt + ((int64_t)h * a.text_rows + drow) * a.D;
+            } else {
+                const int h = slot - a.Hq - a.Hkv;
+                src = a.v + aug * a.v_st + (int64_t)h * a.v_sh;
+                dst = a.vt + ((int64_t)h * a.text_rows + drow) * a.D;
+            }
+        } else {
+            const int64_t drow = (int64_t)sq.summ_off + row;
+            if (slot < a.Hkv) {
+                src = a.kx + aug * a.k_st + (int64_t)slot * a.k_sh;
+                dst = a.ks + ((int64_t)slot * a.summ_rows + drow) * a.D;
+            } else {
+                const int h = slot - a.Hkv;
+                src = a.v + aug * a.v_st + (int64_t)h * a.v_sh;
+                dst = a.vs + ((int64_t)h * a.summ_rows + drow) * a.D;
+            }
+        }
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (row < live_rows) val = *reinterpret_cast<const uint4*>(src + vec * 8);
+        *reinterpret_cast<uint4*>(dst + vec * 8) = val;
+    }
+}
+
+cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream)
+{
+    // grid.x covers the longest padded stream of any sequence (grid-stride loop beyond the cap).
+    const int64_t per_row = (int64_t)(a.Hq + 2 * a.Hkv) * (a.D / 8);
+    const int64_t rows = a.max_text_pad > a.max_summ_pad ? a.max_text_pad : a.max_summ_pad;
+    int64_t blocks = (rows * per_row + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (blocks < 1) blocks = 1;
+    dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, a.m > 0 ? 2u : 1u);
+    ksa_pack_kernel<<<grid, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Summary rows (Sec. 2.2.1, first bullet).  One warp per (summary row, query head): the
+// keys are the contiguous augmented rows j*(k+m) .. j*(k+m) + k - 1 (+ r + 1 own-chunk
+// summaries unless KSA_FLAG_SUMMARY_TEXT_ONLY).  Each lane owns D/32 dimensions.
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
+{
+    constexpr int E = D / 32;
+    const SeqInfo sq = a.seqs[blockIdx.y];
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t total = (int64_t)sq.n_summ * a.Hq;
+    if (warp >= total) return;
+    const int u = (int)(warp / a.Hq);
+    const int h = (int)(warp - (int64_t)u * a.Hq);
+    const int hk = h / (a.Hq / a.Hkv);
+    const int j = u / a.m, r = u - j * a.m;
+    const int s = a.k + a.m;
+    const int64_t key0 = sq.aug_off + (int64_t)j * s;
+    const int64_t qrow = key0 + a.k + r;
+    const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));
+
+    float qv[E], acc[E];
+    {
+        const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) { qv[e] = bf16_bits_to_float(qp[e]); acc[e] = 0.f; }
+    }
+    float mx = -INFINITY, l = 0.f;
+    for (int t = 0; t < nk; ++t) {
+        const uint16_t* kp = a.kx + (key0 + t) * a.k_st + (int64_t)hk * a.k_sh + lane * E;
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) dot = fmaf(qv[e], bf16_bits_to_float(kp[e]), dot);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        const float x = dot * a.scale;
+        const float mn = fmaxf(mx, x);
+        const float alpha = __expf(mx - mn);     // exp(-inf) = 0 on the first key
+        const float p = __expf(x - mn);
+        l = l * alpha + p;
+        const uint16_t* vp = a.v + (key0 + t) * a.v_st + (int64_t)hk * a.v_sh + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = fmaf(acc[e], alpha, p * bf16_bits_to_float(vp[e]));
+        mx = mn;
+    }
+    const float inv = 1.f / l;
+    uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
+    if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
+}
+
+cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
+{
+    if (a.m <= 0 || a.max_n_summ <= 0) return cudaSuccess;
+    // grid.x covers the sequence with the most summary rows; shorter ones exit early.
+    const int64_t warps = (int64_t)a.max_n_summ * a.Hq;
+    int64_t blocks = (warps + 7) / 8;
+    if (blocks < 1) blocks = 1;
+    dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, 1);
+    if (a.D == 128) ksa_summary_kernel<128><<<grid, 256, 0, stream>>>(a);
+    else            ksa_summary_kernel<64><<<grid, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Text rows, cross-check kernel.  One block per work item, one warp per (row, head) in
+// turn.  Walks exactly the tiles the schedule lists, applies the per-row column interval
+// of Eq. 3 inside each tile, fp32 online softmax on CUDA cores.
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) ksa_text_ref_kernel(KernelArgs a)
+{
+    constexpr int E = D / 32;
+    const WorkItem w = a.work[blockIdx.x];
+    const SeqInfo sq = a.seqs[w.seq];
+    const int lane = threadIdx.x & 31;
+    const int nwarps = blockDim.x >> 5;
+    const int s = a.k + a.m;
+    for (int job = threadIdx.x >> 5; job < kTileM * w.n_heads; job += nwarps) {
+        const int rl = job % kTileM;
+        const int h = w.head0 + job / kTileM;
+        const int hk = h / (a.Hq / a.Hkv);
+        const int i = w.q_tile * kTileM + rl;
+        if (i >= sq.n_text) continue;
+        const int c = i / a.k;
+        const int far = max(0, c - a.C);
+        const int lo_i = far * a.k;       // first visible text token
+        const int cnt_i = far * a.m;      // visible summaries: stream rows [0, cnt_i)
+
+        float qv[E], acc[E];
+        const uint16_t* qp = a.qt + ((int64_t)h * a.text_rows + sq.text_off + i) * D + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) { qv[e] = bf16_bits_to_float(qp[e]); acc[e] = 0.f; }
+        float mx = -INFINITY, l = 0.f;
+
+        auto visit = [&](const uint16_t* kbase, const uint16_t* vbase, int c0, int c1) {
+            for (int t = c0; t < c1; ++t) {
+                const uint16_t* kp = kbase + (int64_t)t * D + lane * E;
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) dot = fmaf(qv[e], bf16_bits_to_float(kp[e]), dot);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                const float x = dot * a.scale;
+                const float mn = fmaxf(mx, x);
+                const float alpha = __expf(mx - mn);
+                const float p = __expf(x - mn);
+                l = l * alpha + p;
+                const uint16_t* vp = vbase + (int64_t)t * D + lane * E;
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] = fmaf(acc[e], alpha, p * bf16_bits_to_float(vp[e]));
+                mx = mn;
+            }
+        };
+        {   // summary tiles [0, ns_tiles)
+            const uint16_t* kb = a.ks + ((int64_t)hk * a.summ_rows + sq.summ_off) * D;
+            const uint16_t* vb = a.vs + ((int64_t)hk * a.summ_rows + sq.summ_off) * D;
+            for (int ut = 0; ut < w.ns_tiles; ++ut)
+                visit(kb, vb, ut * kTileN, min(cnt_i, ut * kTileN + kTileN));
+        }
+        {   // text tiles [band_lo, band_hi]
+            const uint16_t* kb = a.kt + ((int64_t)hk * a.text_rows + sq.text_off) * D;
+            const uint16_t* vb = a.vt + ((int64_t)hk * a.text_rows + sq.text_off) * D;
+            for (int bt = w.band_lo; bt <= w.band_hi; ++bt)
+                visit(kb, vb, max(lo_i, bt * kTileN), min(i + 1, bt * kTileN + kTileN));
+        }
+        const float inv = 1.f / l;
+        const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * s + (i % a.k);
+        uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
+        if (lane == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
+    }
+}
+
+cudaError_t launch_text_ref(const KernelArgs& a, cudaStream_t stream)
+{
+    if (a.num_work <= 0) return cudaSuccess;
+    if (a.D == 128) ksa_text_ref_kernel<128><<<a.num_work, 256, 0, stream>>>(a);
+    else            ksa_text_ref_kernel<64><<<a.num_work, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace ksa

@@ -1,0 +1,72 @@
+// Shared host/device declarations of the KSA forward library (internal).
+#pragma once
+#include <stdint.h>
+
+namespace ksa {
+
+constexpr int kTileM = 128;   // query rows per tile
+constexpr int kTileN = 128;   // key/value rows per tile
+
+// Per-sequence layout (Eq. 1): derived once on the host, read by every kernel.
+struct SeqInfo {
+    int64_t aug_off;    // first augmented row of the sequence in q/k/v/out
+    int32_t n_text;     // n_b
+    int32_t n_chunks;   // J_b = floor(n_b / k) full chunks
+    int32_t n_summ;     // J_b * m rows of the summary stream
+    int32_t text_off;   // first row of the sequence in the packed text stream (multiple of kTileM)
+    int32_t summ_off;   // first row in the packed summary stream (multiple of kTileN)
+    int32_t text_pad;   // padded text rows (multiple of kTileM)
+    int32_t summ_pad;   // padded summary rows (multiple of kTileN)
+    int32_t reserved;
+};
+
+// One unit of work of the text-row kernel: one query tile, one or two query heads that
+// share a KV head, and the key/value tiles Eq. 3 makes visible to that tile.
+struct WorkItem {
+    int32_t seq;
+    int32_t q_tile;           // query rows [q_tile*kTileM, +kTileM) of the text stream
+    int32_t head0;            // first query head
+    int32_t n_heads;          // 1 or 2 (head0, head0+1)
+    int32_t ns_tiles;         // summary-stream tiles [0, ns_tiles) are visited
+    int32_t ns_nomask;        // of those, tiles [0, ns_nomask) need no in-tile mask
+    int32_t band_lo, band_hi; // text-stream tiles [band_lo, band_hi] are visited
+    int32_t band_nomask_lo;   // text tiles [band_nomask_lo, band_nomask_hi) need no mask
+    int32_t band_nomask_hi;
+    int32_t reserved0, reserved1;
+};
+static_assert(sizeof(WorkItem) == 48, "WorkItem layout");
+
+// Arguments common to the kernels.
+struct KernelArgs {
+    const SeqInfo* seqs;
+    const WorkItem* work;
+    int32_t num_seqs;
+    int32_t num_work;
+    int32_t k, m, C;
+    int32_t Hq, Hkv, D;
+    uint32_t flags;
+    float scale;            // softmax scale
+    float scale_log2;       // scale * log2(e)
+    int64_t total_aug;
+    int64_t text_rows;      // padded rows of the packed text stream
+    int64_t summ_rows;      // padded rows of the packed summary stream
+    int32_t max_text_pad;   // largest per-sequence padded text rows
+    int32_t max_summ_pad;   // largest per-sequence padded summary rows
+    int32_t max_n_summ;     // largest per-sequence summary count
+    int32_t reserved;
+    // user tensors (bf16 as uint16)
+    const uint16_t* q; const uint16_t* kx; const uint16_t* v; uint16_t* out; float* lse;
+    int64_t q_st, q_sh, k_st, k_sh, v_st, v_sh, o_st, o_sh;
+    // packed streams in the workspace, head-major [H][rows][D]
+    uint16_t* qt; uint16_t* kt; uint16_t* vt; uint16_t* ks; uint16_t* vs;
+    int32_t* status;        // device status word for bounded waits
+};
+
+// Device status codes (which bounded wait gave up first).
+enum DeviceStatus : int32_t {
+    kStatusOk = 0,
+    kStatusWaitQFull = 1, kStatusWaitQEmpty = 2, kStatusWaitKvFull = 3, kStatusWaitKvEmpty = 4,
+    kStatusWaitSFull = 5, kStatusWaitPFull = 6, kStatusWaitOFull = 7, kStatusWaitTest = 8,
+};
+
+}  // namespace ksa

@@ -1,0 +1,27 @@
+// Internal launch interface between the C ABI (ksa_api.cu) and the kernel files.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "ksa_common.h"
+
+namespace ksa {
+
+// De-interleaves text Q/K/V rows and summary K/V rows of the augmented layout (Eq. 1)
+// into dense head-major streams; padding rows are written as zeros.
+cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream);
+
+// Summary rows: each attends to the (at most k + m) keys of its own chunk.
+cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream);
+
+// Text rows, CUDA-core cross-check kernel (KSA_FLAG_REFERENCE_KERNEL).
+cudaError_t launch_text_ref(const KernelArgs& a, cudaStream_t stream);
+
+// Text rows, tcgen05/TMA kernel.  The five tensor maps describe the packed streams
+// as [D, rows, H] with a {64, 128, 1} box and 128-byte swizzle.
+struct TextMaps { CUtensorMap qt, kt, vt, ks, vs; };
+cudaError_t launch_text_tc(const KernelArgs& a, const TextMaps& maps, int num_sms, cudaStream_t stream);
+// One-time per-device setup (dynamic shared memory opt-in).
+cudaError_t setup_text_tc();
+
+}  // namespace ksa

@@ -1,0 +1,438 @@
+// Text-row KSA attention on the sm_100a tensor cores.
+//
+// One persistent CTA per SM walks its share of the work list.  A work item is one tile of
+// 128 text query rows for one or two query heads that share a KV head, plus the key/value
+// tiles Eq. 3 makes visible to it: tiles of the packed summary stream first, then tiles of
+// the packed text stream (the sliding-chunk band up to the diagonal).
+//
+// Warp roles (320 threads):
+//   warps 0-3   softmax of query tile 0 (one row per thread), O rescale, epilogue
+//   warps 4-7   softmax of query tile 1
+//   warp  8     TMA producer: Q tiles, then K and V tiles through a ring of smem stages
+//   warp  9     MMA issuer: S = Q K^T (smem x smem) and O += P V (P from TMEM) via tcgen05.mma
+// TMEM (512 columns): S0 [0,128), S1 [128,256), O0 [256,256+D), O1 [384,384+D); the bf16
+// probabilities P_t overwrite the first 64 columns of S_t.
+//
+// Pipeline per key/value tile j and query tile t:
+//   MMA:     S_t(j) = Q_t K(j)^T                                   -> s_full[t]
+//   softmax: load S_t, mask (only on tiles flagged partial), running max with lazy rescale,
+//            p = 2^(s*scale*log2e - m), row sum, write P_t, rescale O_t if the max moved -> p_full[t]
+//   MMA:     O_t += P_t V(j), then at once S_t(j+1) = Q_t K(j+1)^T -> s_full[t]
+// so that while one query tile is in its softmax the tensor pipe works for the other.
+// tcgen05.mma operations of one thread execute in issue order, which is what lets S_t(j+1)
+// overwrite P_t(j) right after O_t += P_t(j) V(j) was issued, and what makes s_full[t] of
+// tile j imply that O_t += P_t V(j-1) has completed (so the softmax warps may rescale O_t).
+//
+// Every mbarrier wait is bounded: on timeout the thread records which wait gave up in the
+// status word, raises a CTA-wide abort flag, all roles leave their loops, the producer
+// waits (bounded) for its copies in flight, TMEM is freed and the kernel returns.
+#include <cuda_bf16.h>
+
+#include "ksa_launch.h"
+#include "ksa_ptx.cuh"
+
+namespace ksa {
+
+using namespace ptx;
+
+constexpr int kThreadsTc = 320;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr float kRescaleThreshold = 8.0f;    // log2 units: P stays below 2^8
+
+template <int D>
+struct TcCfg {
+    static constexpr int kTileBytes = 128 * D * 2;
+    static constexpr int kHalves = D / 64;                       // 64-column (128-byte) swizzle panels
+    static constexpr int kStages = (D == 128) ? 5 : 10;          // K/V ring depth (tiles)
+    static constexpr int kQOff = 0;
+    static constexpr int kRingOff = 2 * kTileBytes;
+    static constexpr int kBarOff = kRingOff + kStages * kTileBytes;
+    static constexpr int kNumBars = 9 + 2 * kStages;
+    static constexpr int kSmemBytes = kBarOff + 8 * kNumBars + 64 + 1024;   // + slack for 1024-byte alignment
+    // MN-major V operand: the two 64-column panels of a D = 128 tile are 16 KB apart,
+    // groups of 8 keys are 1 KB apart.
+    static constexpr uint32_t kVLbo = 16384;
+    static constexpr uint32_t kVSbo = 1024;
+};
+
+// barrier slots
+enum : int { BAR_QFULL = 0, BAR_QEMPTY = 1, BAR_SFULL = 2, BAR_PFULL = 4, BAR_OFULL = 6, BAR_DRAIN = 8, BAR_KV = 9 };
+
+struct TcShared {
+    uint32_t bars;        // smem address of barrier 0
+    uint32_t abort_addr;  // smem address of the abort flag
+};
+
+__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
+// Bounded wait.  Returns false if the wait gave up or the CTA is aborting.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, uint32_t abort_addr, int32_t* status, int code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (ld_shared_u32(abort_addr) != 0u) return false;
+            if (clock64() - t0 > (1ll << 31)) {
+                atomicCAS(status, 0, code);
+                st_shared_u32(abort_addr, 1u);
+                return false;
+            }
+        }
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__ TextMaps maps)
+{
+    using Cfg = TcCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base + Cfg::kQOff;
+    const uint32_t sRing = smem_base + Cfg::kRingOff;
+    const uint32_t bars = smem_base + Cfg::kBarOff;
+    const uint32_t tmem_slot = bars + 8 * Cfg::kNumBars;
+    const uint32_t abort_addr = tmem_slot + 4;
+    auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+    auto kv_full = [&](int s) -> uint32_t { return bars + 8u * (uint32_t)(BAR_KV + s); };
+    auto kv_empty = [&](int s) -> uint32_t { return bars + 8u * (uint32_t)(BAR_KV + Cfg::kStages + s); };
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    if (tid == 0) {
+        mbar_init(bar(BAR_QFULL), 1);
+        mbar_init(bar(BAR_QEMPTY), 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(BAR_SFULL + t), 1);
+            mbar_init(bar(BAR_PFULL + t), 128);
+            mbar_init(bar(BAR_OFULL + t), 1);
+        }
+        mbar_init(bar(BAR_DRAIN), 1);
+        for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+        st_shared_u32(abort_addr, 0u);
+        st_shared_u32(abort_addr + 4, 0u);     // never raised: lets the teardown waits run while aborting
+        fence_mbar_init();
+    }
+    if (warp == kProducerWarp) {            // one warp allocates all 512 TMEM columns (1 CTA per SM)
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ld_shared_u32(tmem_slot);
+
+    const int G = a.Hq / a.Hkv;
+    const int grid = (int)gridDim.x;
+    const int cta = (int)blockIdx.x;
+    // items are taken in snake order over the longest-first list: round r gives this CTA
+    // item r*grid + cta (even r) or r*grid + grid-1-cta (odd r)
+    auto item_index = [&](int r) -> int { return r * grid + ((r & 1) ? (grid - 1 - cta) : cta); };
+
+    if (warp == kProducerWarp) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            prefetch_tensormap(&maps.qt); prefetch_tensormap(&maps.kt); prefetch_tensormap(&maps.vt);
+            prefetch_tensormap(&maps.ks); prefetch_tensormap(&maps.vs);
+            uint32_t q_phase = 0, ring_phase = 0;
+            int stage = 0;
+            uint32_t armed_mask = 0, armed_parity = 0;   // per stage: a load was issued / with which parity
+            bool q_armed = false;
+            bool alive = true;
+            for (int r = 0; alive; ++r) {
+                const int idx = item_index(r);
+                if (idx >= a.num_work) break;
+                const WorkItem w = a.work[idx];
+                const SeqInfo sq = a.seqs[w.seq];
+                const int hk = w.head0 / G;
+                const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
+                if (!bounded_wait(bar(BAR_QEMPTY), q_phase ^ 1u, abort_addr, a.status, kStatusWaitQEmpty)) break;
+                mbar_arrive_expect_tx(bar(BAR_QFULL), (uint32_t)(w.n_heads * Cfg::kTileBytes));
+                q_armed = true;
+                for (int t = 0; t < w.n_heads; ++t)
+                    for (int h = 0; h < Cfg::kHalves; ++h)
+                        tma_load_3d(sQ + t * Cfg::kTileBytes + h * 16384, &maps.qt, bar(BAR_QFULL),
+                                    h * 64, sq.text_off + w.q_tile * kTileM, w.head0 + t);
+                q_phase ^= 1u;
+                for (int j = 0; j < T && alive; ++j) {
+                    const bool summ = j < w.ns_tiles;
+                    const int y = summ ? (sq.summ_off + j * kTileN) : (sq.text_off + (w.band_lo + j - w.ns_tiles) * kTileN);
+                    const CUtensorMap* mk = summ ? &maps.ks : &maps.kt;
+                    const CUtensorMap* mv = summ ? &maps.vs : &maps.vt;
+                    for (int kv = 0; kv < 2; ++kv) {
+                        if (!bounded_wait(kv_empty(stage), ring_phase ^ 1u, abort_addr, a.status, kStatusWaitKvEmpty)) { alive = false; break; }
+                        mbar_arrive_expect_tx(kv_full(stage), (uint32_t)Cfg::kTileBytes);
+                        armed_mask |= 1u << stage;
+                        armed_parity = (armed_parity & ~(1u << stage)) | (ring_phase << stage);
+                        for (int h = 0; h < Cfg::kHalves; ++h)
+                            tma_load_3d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, y, hk);
+                        if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                    }
+                }
+            }
+            if (ld_shared_u32(abort_addr) != 0u) {
+                // leave no copy in flight behind: wait (bounded) for every load that was issued
+                if (q_armed) bounded_wait(bar(BAR_QFULL), q_phase ^ 1u, abort_addr + 4, a.status, kStatusWaitQFull);
+                for (int s = 0; s < Cfg::kStages; ++s)
+                    if (armed_mask & (1u << s))
+                        bounded_wait(kv_full(s), (armed_parity >> s) & 1u, abort_addr + 4, a.status, kStatusWaitKvFull);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // =============================== MMA issuer =================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
+            uint32_t qf_phase = 0, pf_phase[2] = {0, 0}, ring_phase = 0;
+            int stage = 0;
+            bool alive = true;
+            auto issue_qk = [&](int t, int st) {
+                const uint64_t qd = make_smem_desc_sw128(sQ + t * Cfg::kTileBytes, 16, 1024);
+                const uint64_t kd = make_smem_desc_sw128(sRing + st * Cfg::kTileBytes, 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                    mma_ss(tmem + t * 128, qd + off, kd + off, idesc_qk, kk > 0 ? 1u : 0u);
+                }
+            };
+            auto issue_pv = [&](int t, int st, bool acc) {
+                const uint64_t vd = make_smem_desc_sw128(sRing + st * Cfg::kTileBytes, Cfg::kVLbo, Cfg::kVSbo);
+#pragma unroll
+                for (int kk = 0; kk < kTileN / 16; ++kk)
+                    mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, vd + (uint32_t)((kk * 2048) >> 4), idesc_pv,
+                           (acc || kk > 0) ? 1u : 0u);
+            };
+            for (int r = 0; alive; ++r) {
+                const int idx = item_index(r);
+                if (idx >= a.num_work) break;
+                const WorkItem w = a.work[idx];
+                const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
+                const int nh = w.n_heads;
+                if (!bounded_wait(bar(BAR_QFULL), qf_phase, abort_addr, a.status, kStatusWaitQFull)) break;
+                qf_phase ^= 1u;
+                if (!bounded_wait(kv_full(stage), ring_phase, abort_addr, a.status, kStatusWaitKvFull)) break;
+                tc_fence_after();
+                for (int t = 0; t < nh; ++t) { issue_qk(t, stage); tc_commit(bar(BAR_SFULL + t)); }
+                tc_commit(kv_empty(stage));
+                if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                if (T == 1) tc_commit(bar(BAR_QEMPTY));
+                for (int j = 0; j < T && alive; ++j) {
+                    const int vstage = stage; const uint32_t vphase = ring_phase;
+                    if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                    int kstage = -1; uint32_t kphase = 0;
+                    if (j + 1 < T) {
+                        kstage = stage; kphase = ring_phase;
+                        if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                    }
+                    if (!bounded_wait(kv_full(vstage), vphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                    for (int t = 0; t < nh; ++t) {
+                        if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
+                        pf_phase[t] ^= 1u;
+                        tc_fence_after();
+                        issue_pv(t, vstage, j > 0);
+                        if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
+                        if (j + 1 < T) {
+                            if (t == 0) {
+                                if (!bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                                tc_fence_after();
+                            }
+                            issue_qk(t, kstage);
+                            tc_commit(bar(BAR_SFULL + t));
+                        }
+                    }
+                    if (!alive) break;
+                    tc_commit(kv_empty(vstage));
+                    if (j + 1 < T) {
+                        tc_commit(kv_empty(kstage));
+                        if (j + 1 == T - 1) tc_commit(bar(BAR_QEMPTY));
+                    }
+                }
+            }
+            // drain the tensor pipe before TMEM is released
+            tc_commit(bar(BAR_DRAIN));
+            bounded_wait(bar(BAR_DRAIN), 0, abort_addr + 4, a.status, kStatusWaitOFull);
+        }
+    } else {
+        // =============================== softmax warpgroups =========================
+        const int t = warp >> 2;
+        const int row = tid & 127;
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_sel + (uint32_t)(t * 128);
+        const uint32_t tO = tmem + lane_sel + 256u + (uint32_t)(t * 128);
+        const float scale_log2 = a.scale_log2;
+        uint32_t sf_phase = 0, of_phase = 0;
+        const int s_len = a.k + a.m;
+        bool alive = true;
+        for (int r = 0; alive; ++r) {
+            const int idx = item_index(r);
+            if (idx >= a.num_work) break;
+            const WorkItem w = a.work[idx];
+            if (t >= w.n_heads) continue;
+            const SeqInfo sq = a.seqs[w.seq];
+            const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
+            const int i_raw = w.q_tile * kTileM + row;
+            const bool valid = i_raw < sq.n_text;
+            const int i = valid ? i_raw : sq.n_text - 1;     // padding rows mimic the last row; never stored
+            const int chunk = i / a.k;
+            const int far = max(0, chunk - a.C);
+            const int lo_i = far * a.k;                      // Eq. 3: first visible text token
+            const int cnt_i = far * a.m;                     // Eq. 3: summaries [0, cnt_i) visible
+            float m_used = -INFINITY, l_run = 0.f;
+
+            for (int j = 0; j < T; ++j) {
+                bool ok = bounded_wait(bar(BAR_SFULL + t), sf_phase, abort_addr, a.status, kStatusWaitSFull);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { alive = false; break; }
+                sf_phase ^= 1u;
+                tc_fence_after();
+                uint32_t s[128];
+                {
+                    uint32_t (&c0)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[0]);
+                    uint32_t (&c1)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[32]);
+                    uint32_t (&c2)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[64]);
+                    uint32_t (&c3)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[96]);
+                    tmem_ld32(tS + 0, c0); tmem_ld32(tS + 32, c1); tmem_ld32(tS + 64, c2); tmem_ld32(tS + 96, c3);
+                }
+                tc_wait_ld();
+                // in-tile mask, only where the schedule says the tile is partial
+                bool masked;
+                int ca, cb;                                   // visible columns [ca, cb)
+                if (j < w.ns_tiles) {
+                    masked = j >= w.ns_nomask;
+                    ca = 0; cb = cnt_i - j * kTileN;
+                } else {
+                    const int bt = w.band_lo + (j - w.ns_tiles);
+                    masked = !(bt >= w.band_nomask_lo && bt < w.band_nomask_hi);
+                    ca = lo_i - bt * kTileN; cb = i + 1 - bt * kTileN;
+                }
+                if (masked) {
+                    const uint32_t width = (uint32_t)max(cb - ca, 0);
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if ((uint32_t)(c - ca) >= width) s[c] = 0xff800000u;   // -inf
+                }
+                float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
+                float mx2 = __uint_as_float(s[2]), mx3 = __uint_as_float(s[3]);
+#pragma unroll
+                for (int c = 4; c < 128; c += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[c]));     mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+                }
+                const float mx_sc = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
+                // lazy rescale: the reference max only moves when some row of the warp outgrew it
+                const bool need = mx_sc > m_used + kRescaleThreshold;
+                const bool need_any = __any_sync(0xffffffffu, need);
+                float alpha = 1.f;
+                if (need_any) {
+                    const float m_new = fmaxf(m_used, mx_sc);
+                    alpha = (m_new == -INFINITY) ? 1.f : ex2_approx(m_used - m_new);
+                    m_used = m_new;
+                    l_run *= alpha;
+                }
+                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+                for (int c = 0; c < 128; c += 4) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), scale_log2, neg_m));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), scale_log2, neg_m));
+                    const float p2 = ex2_approx(fmaf(__uint_as_float(s[c + 2]), scale_log2, neg_m));
+                    const float p3 = ex2_approx(fmaf(__uint_as_float(s[c + 3]), scale_log2, neg_m));
+                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                    s[c / 2] = pack_bf16x2(p0, p1);
+                    s[c / 2 + 1] = pack_bf16x2(p2, p3);
+                }
+                l_run += (l0 + l1) + (l2 + l3);
+                {
+                    uint32_t (&p0)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[0]);
+                    uint32_t (&p1)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[32]);
+                    tmem_st32(tS + 0, p0); tmem_st32(tS + 32, p1);
+                }
+                if (need_any && j > 0) {
+                    // O_t += P V(j-1) has completed (s_full of tile j was committed after it)
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(BAR_PFULL + t));
+            }
+            if (!alive) break;
+            // ---- epilogue: O / l -> bf16 at the row's augmented position (Eq. 1), LSE ----
+            bool ok = bounded_wait(bar(BAR_OFULL + t), of_phase, abort_addr, a.status, kStatusWaitOFull);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            of_phase ^= 1u;
+            tc_fence_after();
+            const float inv_l = 1.f / l_run;
+            const int h = w.head0 + t;
+            const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * s_len + (i % a.k);
+            uint16_t* orow = a.out + aug * a.o_st + (int64_t)h * a.o_sh;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                tc_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 pk;
+                        pk.x = pack_bf16x2(__uint_as_float(o[e]) * inv_l, __uint_as_float(o[e + 1]) * inv_l);
+                        pk.y = pack_bf16x2(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
+                        pk.z = pack_bf16x2(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
+                        pk.w = pack_bf16x2(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + e) = pk;
+                    }
+                }
+            }
+            if (valid) a.lse[(int64_t)h * a.total_aug + aug] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+            tc_fence_before();
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kProducerWarp) tmem_dealloc(tmem, 512);
+}
+
+cudaError_t setup_text_tc()
+{
+    cudaError_t e = cudaFuncSetAttribute(ksa_text_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TcCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(ksa_text_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TcCfg<64>::kSmemBytes);
+}
+
+cudaError_t launch_text_tc(const KernelArgs& a, const TextMaps& maps, int num_sms, cudaStream_t stream)
+{
+    if (a.num_work <= 0) return cudaSuccess;
+    const int grid = a.num_work < num_sms ? a.num_work : num_sms;
+    if (a.D == 128)
+        ksa_text_tc_kernel<128><<<grid, kThreadsTc, TcCfg<128>::kSmemBytes, stream>>>(a, maps);
+    else
+        ksa_text_tc_kernel<64><<<grid, kThreadsTc, TcCfg<64>::kSmemBytes, stream>>>(a, maps);
+    return cudaGetLastError();
+}
+
+}  // namespace ksa

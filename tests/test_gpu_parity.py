@@ -1,0 +1,141 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ksa_oracle as orc
+from paper_2604_24432_b200 import binding as ksa
+from paper_2604_24432_b200 import build as ksa_build
+from paper_2604_24432_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+REF = ksa.KSA_FLAG_REFERENCE_KERNEL
+STRICT = ksa.KSA_FLAG_SUMMARY_TEXT_ONLY
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    ksa_build.build()
+    c = ksa.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
+@pytest.mark.parametrize("layout", [synth.LAYOUT_P, synth.LAYOUT_G], ids=["P", "G"])
+@pytest.mark.parametrize("C", [None, 0, 1, 2, 4])
+def test_tiny_full(ctx, kernel_flag, layout, C):
+    """1,024 text tokens, 4/4 heads, D = 64: every row against the oracle, at the paper's
+    window (pure causal over text) and at small windows that make summaries visible."""
+    parity.check_workload(ctx, synth.WORKLOADS["tiny"], layout, kernel_flag, C=C)
+
+
+@pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
+def test_tiny_strict_summary_rule(ctx, kernel_flag):
+    parity.check_workload(ctx, synth.WORKLOADS["tiny"], synth.LAYOUT_G, kernel_flag | STRICT, C=2)
+    parity.check_workload(ctx, synth.WORKLOADS["tiny"], synth.LAYOUT_P, kernel_flag | STRICT, C=2)
+
+
+@pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
+def test_8k_full(ctx, kernel_flag):
+    """8,192 text tokens, GQA 32/8, D = 128, K scaled by 0.5 (flat softmax): every row."""
+    parity.check_workload(ctx, synth.WORKLOADS["8k"], synth.LAYOUT_P, kernel_flag)
+
+
+def test_8k_layout_g_sampled(ctx):
+    parity.check_workload(ctx, synth.WORKLOADS["8k"], synth.LAYOUT_G, 0, n_random=512, seed=1)
+
+
+@pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
+    ([1], 8, 1, 2, 2, 2, 64),              # a single token
+    ([7], 8, 1, 2, 2, 1, 128),             # shorter than a chunk: no summary at all
+    ([127, 129, 128], 8, 1, 3, 4, 2, 64),  # ragged tiles, packed
+    ([333, 1000], 3, 2, 5, 6, 2, 128),     # k does not divide the tile, m = 2, G = 3 (one head per item)
+    ([777], 16, 0, 7, 4, 4, 64),           # m = 0: sliding chunk attention alone (Eq. 2)
+    ([640], 1, 1, 100, 2, 1, 128),         # k = 1
+    ([1290], 200, 3, 1, 4, 1, 128),        # chunk longer than a tile
+    ([2100], 8, 1, 16, 8, 2, 128),         # several summary tiles
+])
+def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
+    wl = synth.Workload("edge", 99, lens, Hq, Hkv, D)
+    parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), kernel_flag)
+
+
+def test_strided_inputs_and_stream(ctx):
+    """Non-contiguous q/k/v/out views (packed QKV buffer) on a side stream."""
+    wl = synth.Workload("strided", 5, [900], 8, 2, 128)
+    lay = synth.Layout("s", 8, 1, 4)
+    total = orc.aug_len(900, 8, 1)
+    q, k, v = synth.make_qkv(wl, total)
+    dev = torch.device("cuda", 0)
+    packed = torch.zeros((total, 8 + 2 + 2 + 1, 128), dtype=torch.bfloat16, device=dev)
+    packed[:, :8] = q.to(dev); packed[:, 8:10] = k.to(dev); packed[:, 10:12] = v.to(dev)
+    qd, kd, vd = packed[:, :8], packed[:, 8:10], packed[:, 10:12]
+    outbuf = torch.zeros((total, 9, 128), dtype=torch.bfloat16, device=dev)
+    out = outbuf[:, 1:]
+    lse = torch.empty((8, total), dtype=torch.float32, device=dev)
+    prob = ksa.Problem([900], 8, 1, 4, 8, 2, 128, wl.scale)
+    ws = torch.empty(ksa.workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws, stream=st.cuda_stream)
+    st.synchronize()
+    ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), [900], 8, 1, 4, wl.scale)
+    parity.compare(out.double().cpu().numpy(), lse.double().cpu().numpy().T, ref_out, ref_lse, "strided")
+    assert (outbuf[:, 0] == 0).all()
+
+
+def test_host_entry_point(ctx):
+    wl = synth.Workload("host", 6, [500, 300], 4, 2, 128)
+    total = orc.aug_len(500, 8, 1) + orc.aug_len(300, 8, 1)
+    q, k, v = synth.make_qkv(wl, total, pin=True)
+    prob = ksa.Problem([500, 300], 8, 1, 2, 4, 2, 128, wl.scale)
+    out = torch.empty((total, 4, 128), dtype=torch.bfloat16).pin_memory()
+    lse = torch.empty((4, total), dtype=torch.float32).pin_memory()
+    staging = torch.empty(ksa.host_staging_bytes(prob), dtype=torch.uint8, device="cuda:0")
+    ctx.attn_fwd_host(prob, q, k, v, out, lse, staging)
+    ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), [500, 300], 8, 1, 2, wl.scale)
+    parity.compare(out.double().numpy(), lse.double().numpy().T, ref_out, ref_lse, "host")
+
+
+def test_runtime_argument_errors(ctx):
+    dev = torch.device("cuda", 0)
+    prob = ksa.Problem([300], 8, 1, 2, 4, 2, 64, 0.125)
+    total = ksa.total_aug_len(prob)
+    q = torch.zeros((total, 4, 64), dtype=torch.bfloat16, device=dev)
+    k = torch.zeros((total, 2, 64), dtype=torch.bfloat16, device=dev)
+    out = torch.zeros_like(q)
+    lse = torch.zeros((4, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(ksa.workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    before = ctx.launch_count()
+    with pytest.raises(ksa.KsaError) as e:
+        ctx.attn_fwd(prob, q, k, k, out, lse, ws[:1024])
+    assert e.value.status == ksa.KSA_ERR_WORKSPACE
+    with pytest.raises(ksa.KsaError) as e:
+        ctx.attn_fwd(prob, q.view(-1)[1:].view(-1)[: (total - 1) * 256].view(total - 1, 4, 64), k, k, out, lse, ws)
+    assert e.value.status == ksa.KSA_ERR_INVALID_ARG     # misaligned q
+    bad = dataclasses.replace(prob, k=0)
+    with pytest.raises(ksa.KsaError):
+        ctx.attn_fwd(bad, q, k, k, out, lse, ws)
+    assert ctx.launch_count() == before                  # nothing was launched
+    ctx.attn_fwd(prob, q, k, k, out, lse, ws)
+    torch.cuda.synchronize()
+    assert ctx.launch_count() == before + 3
+
+
+def test_q_zero_gives_log_count(ctx):
+    """Q = 0: lse = ln(visible count) and out = mean of the visible V rows, for every row."""
+    wl = synth.Workload("q0", 7, [1500], 4, 2, 128)
+    lay = synth.Layout("q0", 8, 1, 16)
+    total = orc.aug_len(1500, 8, 1)
+    q, k, v = synth.make_qkv(wl, total)
+    q.zero_()
+    prob = ksa.Problem([1500], 8, 1, 16, 4, 2, 128, wl.scale)
+    out, lse = parity.run_gpu(ctx, prob, q, k, v)
+    cnt = np.array([orc.visible_count(1500, 8, 1, 16, p) for p in range(total)])
+    assert np.abs(lse - np.log(cnt)[:, None]).max() < 1e-4
