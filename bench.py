@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the KSA attention forward hot path on B200.
+
+A "step" is one pass of the whole hot path (pack -> summary-row kernel -> text-row
+tensor-core kernel) over one batch of synthetic input shaped like the paper's 128K
+long-context workload (131,072 text tokens, chunk size 8 with one summary token, 128
+sliding chunks, GQA 32/4, head dim 128, bf16).  The metric is visible TFLOP/s: only the
+(query, key) pairs the KSA mask makes visible count, 4*D flops each per query head.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 128k] [--layout P]
+    python bench.py --impl reference ...      # the CPU oracle on a bounded row sample
+
+N > 1 (under torchrun): every rank runs its own independent batch (weak scaling, no
+data-path collective); the value is the aggregate over ranks, timed as max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2604_24432_b200 import synth
+
+METRIC = "KSA attn fwd visible TFLOP/s & text tok/s at 128K, % of B200 BF16 peak"
+
+# DRAM bytes (read + write) of one launch of the text-row kernel at the 128k / P workload,
+# from an ncu capture (see profiles/); None until a capture exists for the current kernel.
+NCU_TEXT_KERNEL_DRAM_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(source="measured", hbm_gbs=float(d["hbm_gbs"]), bf16_burst=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])))
+    return dict(source="fallback", hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, index: int, period: float = 0.05):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                mask = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml_unavailable"]}
+        reasons = sorted(self.reasons - {"gpu_idle"})
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "reasons": reasons}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def workload_and_layout(args):
+    wl = synth.WORKLOADS[args.workload]
+    layout = synth.LAYOUT_P if args.layout == "P" else synth.LAYOUT_G
+    return wl, layout
+
+
+def base_config(wl, layout, world):
+    return {
+        "workload": f"{wl.name} ({wl.note})", "layout": f"{layout.name}: k={layout.k} m={layout.m} C={layout.C}",
+        "text_tokens_per_gpu": int(sum(wl.text_lens)), "heads": f"{wl.Hq}q/{wl.Hkv}kv", "head_dim": wl.D,
+        "l2_policy": "inputs larger than L2 (no flush)", "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+    }
+
+
+# ---------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of rows per step
+# ---------------------------------------------------------------------------------------
+def oracle_sample_rows(wl, layout, n_rows, seed):
+    from oracle import ksa_oracle as orc
+    total = sum(orc.aug_len(n, layout.k, layout.m) for n in wl.text_lens)
+    rng = np.random.default_rng(seed)
+    return np.sort(rng.choice(total, size=min(n_rows, total), replace=False)).astype(np.int64), total
+
+
+def time_oracle(wl, layout, q, k, v, rows):
+    from oracle import ksa_oracle as orc
+    t0 = time.perf_counter()
+    _, _, cnt = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), wl.text_lens, layout.k, layout.m,
+                        layout.C, wl.scale, rows=rows)
+    dt = time.perf_counter() - t0
+    flops = 4.0 * wl.D * wl.Hq * float(cnt.sum())
+    return dt, flops, orc.num_threads()
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    wl, layout = workload_and_layout(args)
+    rows, total = oracle_sample_rows(wl, layout, args.oracle_rows, 1234)
+    q, k, v = synth.make_qkv(wl, total)
+    times, flops = [], 0.0
+    cores = 0
+    for it in range(args.warmup + args.steps):
+        dt, flops, cores = time_oracle(wl, layout, q, k, v, rows)
+        if it >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = flops / (ms * 1e-3) / 1e12
+    sample = f"{len(rows)} random augmented rows of the workload per step, all {wl.Hq} heads"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded, bf16 inputs)",
+        "config": base_config(wl, layout, 1),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2604_24432_b200 import binding as ksa
+    from paper_2604_24432_b200 import build as ksa_build
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0 or world > 1:
+        ksa_build.build()
+    wl, layout = workload_and_layout(args)
+    if world > 1:   # independent batch per rank
+        import dataclasses
+        wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total = ksa.total_aug_len(prob)
+    pairs = ksa.visible_pairs(prob)
+    flops = 4.0 * wl.D * wl.Hq * pairs
+    n_text = int(sum(wl.text_lens))
+
+    qh, kh, vh = synth.make_qkv(wl, total, pin=True)
+    q, k, v = qh.to(dev), kh.to(dev), vh.to(dev)
+    out = torch.empty((total, wl.Hq, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(ksa.workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    ctx = ksa.Context(local)
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        ctx.attn_fwd(prob, q, k, v, out, lse, ws)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0, "device-side wait gave up"
+    ctx.enable_kernel_timing(True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    text_ms = []
+    launches0 = ctx.launch_count()
+    barrier()
+    with ClockSampler(local) as clocks:
+        ev[0].record(stream)
+        for i in range(args.steps):
+            ctx.attn_fwd(prob, q, k, v, out, lse, ws)
+            ev[i + 1].record(stream)
+            # the library's own event pair brackets the text-row kernel of this step
+            text_ms.append(ctx.text_kernel_ms())
+        barrier()
+    launches = ctx.launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    ctx.enable_kernel_timing(False)
+    assert ctx.device_status() == 0, "device-side wait gave up"
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    tok_s = world * n_text / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host entry point ----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        out_h = torch.empty((total, wl.Hq, wl.D), dtype=torch.bfloat16).pin_memory()
+        lse_h = torch.empty((wl.Hq, total), dtype=torch.float32).pin_memory()
+        del out, lse, ws
+        staging = torch.empty(ksa.host_staging_bytes(prob), dtype=torch.uint8, device=dev)
+        ctx.attn_fwd_host(prob, qh, kh, vh, out_h, lse_h, staging)       # warm-up
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            ctx.attn_fwd_host(prob, qh, kh, vh, out_h, lse_h, staging)
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2
+        d2h = out_h.numel() * 2 + lse_h.numel() * 4
+        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
+               "api": "ksa_attn_fwd_host (pinned host tensors)"}
+
+    if rank != 0:
+        return 0
+
+    # ---- roofline of the dominant kernel (text rows, tensor-bound) ------------------------
+    peaks = load_peaks()
+    text_pairs = pairs - summary_pairs(wl, layout)
+    text_flops = 4.0 * wl.D * wl.Hq * text_pairs
+    text_avg_ms = sum(text_ms) / len(text_ms)
+    achieved = text_flops / (text_avg_ms * 1e-3) / 1e12
+    traffic = NCU_TEXT_KERNEL_DRAM_BYTES.get((wl.name, layout.name))
+    roofline = {
+        "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+        "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
+        "peak_source": f"of {peaks['source']} (sustained bf16 GEMM; kernel timed inside a multi-step loop)",
+        "frac_of_burst_peak": achieved / peaks["bf16_burst"], "burst_peak": peaks["bf16_burst"],
+        "kernel": "ksa_text_tc_kernel", "kernel_ms_avg": text_avg_ms, "kernel_share_of_step": text_avg_ms / ms_per_step,
+    }
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only) -----------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        rows, _ = oracle_sample_rows(wl, layout, args.oracle_rows, 1234)
+        dt, oflops, cores = time_oracle(wl, layout, qh, kh, vh, rows)
+        cpu = {"value": oflops / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+               "sample": f"{len(rows)} random augmented rows, all {wl.Hq} heads, {dt:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)",
+        "config": base_config(wl, layout, world),
+        "text_tok_per_s": tok_s, "visible_tflop_per_step": flops / 1e12,
+        "pct_of_peak": {"measured_burst": 100 * value / world / peaks["bf16_burst"],
+                        "measured_sustained": 100 * value / world / peaks["bf16_sustained"],
+                        "nominal_2250": 100 * value / world / 2250.0, "source": peaks["source"]},
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def summary_pairs(wl, layout):
+    """Visible pairs of the summary rows (they run in their own small kernel)."""
+    tot = 0
+    for n in wl.text_lens:
+        J = n // layout.k
+        tot += J * sum(layout.k + r + 1 for r in range(layout.m))
+    return tot
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="128k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--layout", default="P", choices=["P", "G"])
+    ap.add_argument("--oracle-rows", type=int, default=3000)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
