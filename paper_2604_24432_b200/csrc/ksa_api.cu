@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "../../include/ksa.h"
+#include "ksa_host.h"
 #include "ksa_launch.h"
 
 using namespace ksa;
@@ -22,13 +23,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
-struct HostSchedule {
-    std::vector<int32_t> key;         // lengths and parameters this schedule was built for
-    std::vector<SeqInfo> seqs;
-    std::vector<WorkItem> work;       // sorted, longest first
-    int64_t total_aug = 0, text_rows = 0, summ_rows = 0;
-    int32_t max_text_pad = 0, max_summ_pad = 0, max_n_summ = 0;
-};
 
 struct ksa_ctx {
     int device = -1;
@@ -55,7 +49,7 @@ static int cuda_fail(ksa_ctx* ctx, cudaError_t e)
 // ---------------------------------------------------------------------------------------
 // validation and layout
 // ---------------------------------------------------------------------------------------
-static int validate(const ksa_params* p)
+int validate(const ksa_params* p)
 {
     if (!p || p->struct_size != (int32_t)sizeof(ksa_params)) return KSA_ERR_INVALID_ARG;
     if (p->num_seqs < 1 || !p->cu_text_lens) return KSA_ERR_INVALID_ARG;
@@ -79,7 +73,7 @@ static int validate(const ksa_params* p)
     return KSA_OK;
 }
 
-static int validate_strides(const ksa_params* p)
+int validate_strides(const ksa_params* p)
 {
     const int64_t st[8] = {p->q_stride_tok, p->q_stride_head, p->k_stride_tok, p->k_stride_head,
                            p->v_stride_tok, p->v_stride_head, p->o_stride_tok, p->o_stride_head};
@@ -90,7 +84,7 @@ static int validate_strides(const ksa_params* p)
 
 static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
-static void build_layout(const ksa_params* p, HostSchedule& hs)
+void build_layout(const ksa_params* p, HostSchedule& hs)
 {
     const int k = p->chunk_len, m = p->summaries_per_chunk;
     hs.seqs.resize(p->num_seqs);
@@ -187,7 +181,7 @@ static BaseItem schedule_q_tile(const Eq3& e, const SeqInfo& s, int seq, int qt)
     return it;
 }
 
-static void build_schedule(const ksa_params* p, HostSchedule& hs)
+void build_schedule(const ksa_params* p, HostSchedule& hs)
 {
     const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
     const int G = p->num_q_heads / p->num_kv_heads;
@@ -225,8 +219,7 @@ static std::vector<int32_t> schedule_key(const ksa_params* p)
     return key;
 }
 
-struct WorkspaceLayout { size_t qt, kt, vt, ks, vs, total; };
-static WorkspaceLayout workspace_layout(const ksa_params* p, const HostSchedule& hs)
+WorkspaceLayout workspace_layout(const ksa_params* p, const HostSchedule& hs)
 {
     WorkspaceLayout w{};
     const size_t D2 = (size_t)p->head_dim * 2;
