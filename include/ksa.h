@@ -152,6 +152,43 @@ int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, cons
                       void* out_host, float* lse_host, void* staging, size_t staging_bytes,
                       const ksa_params* p, void* cuda_stream);
 
+/* ---- forward without device allocation -------------------------------------------------- */
+/*
+ * (No counterpart in the paper: this is a packaging variant of ksa_attn_fwd.)
+ *
+ * Some programs that want this operator are not allowed to obtain device memory at the
+ * moment they call it: an inference server whose whole GPU has been handed to its own
+ * memory pool at start-up, so that a raw cudaMalloc from a plug-in fails or is forbidden
+ * by policy; a latency-critical loop that cannot tolerate the device-wide
+ * synchronisation cudaMalloc/cudaFree imply; a component that simply has no allocator
+ * handle to pass down.  ksa_create (device tables) and the caller-provided workspace of
+ * ksa_attn_fwd both presuppose an allocator.  This entry point presupposes none: it
+ * needs no context and no workspace, and calls neither cudaMalloc nor cudaFree nor any
+ * other allocating routine.  All of its scratch -- the status word of the bounded waits,
+ * the sequence table, the work list and the packed Q/K/V streams -- lives in one
+ * fixed-size array in the library's device image, KSA_NOALLOC_MAX_SCRATCH_BYTES long,
+ * which every GPU that loads the library holds from load until the process exits.
+ *
+ * Arguments q, k, v, out, lse, p, cuda_stream: exactly as for ksa_attn_fwd, on the
+ * CURRENT device; results are identical to ksa_attn_fwd's.
+ * Limits and behaviour:
+ *   - Problems whose scratch exceeds the array are rejected with KSA_ERR_WORKSPACE
+ *     before anything is enqueued (scratch = 256 B + 48 B per sequence + 48 B per work
+ *     item + ksa_workspace_bytes(p)).
+ *   - The first call on each device resolves the array's device address and opts the
+ *     kernels into their shared-memory size; make that first call outside any stream
+ *     capture.
+ *   - The call uploads its tables with cudaMemcpyAsync and waits for the stream once
+ *     before launching, so it is not fully asynchronous.
+ *   - All calls in a process share the one array per device and the array keeps the
+ *     previous call's contents (the call re-zeroes what must start at zero).  Two calls
+ *     whose GPU work overlaps -- different streams, or different host threads -- race on
+ *     it: serialise them.
+ */
+#define KSA_NOALLOC_MAX_SCRATCH_BYTES (32u * 1024u * 1024u)
+int ksa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
+                         const ksa_params* p, void* cuda_stream);
+
 /* ---- schedule inspection ------------------------------------------------------------ */
 /*
  * Lists every (query tile, key/value tile) pair the text-row kernel visits for p, in

@@ -27,6 +27,7 @@ KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
 EXPORTS = [
     "ksa_create", "ksa_destroy", "ksa_aug_len", "ksa_total_aug_len", "ksa_workspace_bytes",
     "ksa_visible_pairs", "ksa_attn_fwd", "ksa_host_staging_bytes", "ksa_attn_fwd_host",
+    "ksa_attn_fwd_noalloc",
     "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
     "ksa_last_cuda_error", "ksa_launch_count", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
     "ksa_strerror",
@@ -86,6 +87,7 @@ def lib():
     L.ksa_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_host_staging_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
+    L.ksa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, pp, vp]
     L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
     L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.ksa_clear_device_status.argtypes = [vp]
@@ -254,6 +256,21 @@ class Context:
         ms = ctypes.c_float()
         _check(lib().ksa_text_kernel_ms(self.handle, ctypes.byref(ms)), "ksa_text_kernel_ms")
         return float(ms.value)
+
+
+NOALLOC_MAX_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def attn_fwd_noalloc(prob: Problem, q, k, v, out, lse, stream: Optional[int] = None):
+    """ksa_attn_fwd_noalloc: the forward pass for callers that may not allocate device
+    memory (no context, no workspace; the library's fixed internal scratch is used).
+    q, k, v, out, lse are torch CUDA tensors on the current device, owned by the caller."""
+    import torch
+    p = prob.params(q, k, v, out)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    _check(lib().ksa_attn_fwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                      lse.data_ptr(), ctypes.byref(p), stream), "ksa_attn_fwd_noalloc")
 
 
 def attn_fwd(ctx: Context, prob: Problem, q, k, v):
