@@ -50,6 +50,19 @@ def test_8k_layout_g_sampled(ctx):
     parity.check_workload(ctx, synth.WORKLOADS["8k"], synth.LAYOUT_G, 0, n_random=512, seed=1)
 
 
+@pytest.mark.parametrize("name,n_random", [("32k", 768), ("128k", 512), ("varlen", 1024)])
+def test_full_size_sampled(ctx, name, n_random):
+    """The three large workloads at full size, in the launch configuration the benchmark times:
+    every row of the first, last and a few boundary query tiles of each sequence plus random
+    rows, all heads, against the oracle (which computes the sampled rows one by one)."""
+    parity.check_workload(ctx, synth.WORKLOADS[name], synth.LAYOUT_P, 0, n_random=n_random, seed=11)
+
+
+def test_full_size_layout_g_sampled(ctx):
+    """128K at the 64 + 8 chunk layout (m = 8 summaries per chunk), sampled rows."""
+    parity.check_workload(ctx, synth.WORKLOADS["128k"], synth.LAYOUT_G, 0, n_random=256, seed=12)
+
+
 @pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
 @pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
     ([1], 8, 1, 2, 2, 2, 64),              # a single token
