@@ -5,7 +5,7 @@
 // tiles Eq. 3 makes visible to it: tiles of the packed summary stream first, then tiles of
 // the packed text stream (the sliding-chunk band up to the diagonal).
 //
-// Warp roles (320 threads):
+// Warp roles (384 threads = three warpgroups; warps 10-11 idle, they complete the third one):
 //   warps 0-3   softmax of query tile 0 (one row per thread), O rescale, epilogue
 //   warps 4-7   softmax of query tile 1
 //   warp  8     TMA producer: Q tiles, then K and V tiles through a ring of smem stages
@@ -35,7 +35,26 @@ namespace ksa {
 
 using namespace ptx;
 
-constexpr int kThreadsTc = 320;
+// Optional event trace (compile with -DKSA_TRACE): CTAs 0 and 100 record (event id, clock) pairs
+// per role into a device buffer that ksa_debug_read_trace() copies out.  Compiled out by default.
+#ifdef KSA_TRACE
+constexpr int kTraceEvents = 8192;
+__device__ uint2 g_trace[2][4][kTraceEvents];
+__device__ uint32_t g_trace_cnt[2][4];
+#define KSA_TR(role, id)                                                                           \
+    do {                                                                                           \
+        if (tr_slot >= 0 && tr_n < (uint32_t)kTraceEvents) {                                       \
+            g_trace[tr_slot][role][tr_n] = make_uint2((uint32_t)(id), (uint32_t)clock64());        \
+            g_trace_cnt[tr_slot][role] = ++tr_n;                                                   \
+        }                                                                                          \
+    } while (0)
+#else
+#define KSA_TR(role, id) do { } while (0)
+#endif
+
+constexpr int kThreadsTc = 384;           // three warpgroups; warps 10 and 11 only take part in the register hand-over
+constexpr int kRegsSoftmax = 216;         // registers per thread of the softmax warpgroups after the hand-over
+constexpr int kRegsOther = 72;            // ... of the producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;    // log2 units: P stays below 2^8
@@ -112,13 +131,17 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+#ifdef KSA_TRACE
+    const int tr_slot = (blockIdx.x == 0) ? 0 : ((blockIdx.x == 100) ? 1 : -1);
+    uint32_t tr_n = 0;
+#endif
 
     if (tid == 0) {
         mbar_init(bar(BAR_QFULL), 1);
         mbar_init(bar(BAR_QEMPTY), 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(BAR_SFULL + t), 1);
-            mbar_init(bar(BAR_PFULL + t), 128);
+            mbar_init(bar(BAR_PFULL + t), 4);      // one arrival per softmax warp
             mbar_init(bar(BAR_OFULL + t), 1);
         }
         mbar_init(bar(BAR_DRAIN), 1);
@@ -143,6 +166,10 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
     // item r*grid + cta (even r) or r*grid + grid-1-cta (odd r)
     auto item_index = [&](int r) -> int { return r * grid + ((r & 1) ? (grid - 1 - cta) : cta); };
 
+    if (warp >= 8) {
+    // register hand-over: this warpgroup gives most of its registers to the softmax warpgroups,
+    // which keep a whole 128-column score row per thread
+    setmaxnreg_dec<kRegsOther>();
     if (warp == kProducerWarp) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
@@ -242,6 +269,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     for (int t = 0; t < nh; ++t) {
                         if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
                         pf_phase[t] ^= 1u;
+                        KSA_TR(0, 20 + t);
                         tc_fence_after();
                         issue_pv(t, vstage, j > 0);
                         if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
@@ -252,6 +280,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                             }
                             issue_qk(t, kstage);
                             tc_commit(bar(BAR_SFULL + t));
+                            KSA_TR(0, 30 + t);
                         }
                     }
                     if (!alive) break;
@@ -266,7 +295,9 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             tc_commit(bar(BAR_DRAIN));
             bounded_wait(bar(BAR_DRAIN), 0, abort_addr + 4, a.status, kStatusWaitOFull);
         }
+    }
     } else {
+        setmaxnreg_inc<kRegsSoftmax>();
         // =============================== softmax warpgroups =========================
         const int t = warp >> 2;
         const int row = tid & 127;
@@ -298,6 +329,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { alive = false; break; }
                 sf_phase ^= 1u;
+                if (row == 0) KSA_TR(1 + t, 1);
                 tc_fence_after();
                 uint32_t s[128];
                 {
@@ -308,6 +340,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     tmem_ld32(tS + 0, c0); tmem_ld32(tS + 32, c1); tmem_ld32(tS + 64, c2); tmem_ld32(tS + 96, c3);
                 }
                 tc_wait_ld();
+                if (row == 0) KSA_TR(1 + t, 2);
                 // in-tile mask, only where the schedule says the tile is partial
                 bool masked;
                 int ca, cb;                                   // visible columns [ca, cb)
@@ -325,14 +358,22 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     for (int c = 0; c < 128; ++c)
                         if ((uint32_t)(c - ca) >= width) s[c] = 0xff800000u;   // -inf
                 }
-                float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
-                float mx2 = __uint_as_float(s[2]), mx3 = __uint_as_float(s[3]);
+                // row maximum, two new scores per instruction
+                float mx0 = fmax3(__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]));
+                float mx1 = fmax3(__uint_as_float(s[3]), __uint_as_float(s[4]), __uint_as_float(s[5]));
+                float mx2 = fmax3(__uint_as_float(s[6]), __uint_as_float(s[7]), __uint_as_float(s[8]));
+                float mx3 = fmax3(__uint_as_float(s[9]), __uint_as_float(s[10]), __uint_as_float(s[11]));
 #pragma unroll
-                for (int c = 4; c < 128; c += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[c]));     mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+                for (int c = 12; c < 124; c += 8) {
+                    mx0 = fmax3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
                 }
+                mx0 = fmax3(mx0, __uint_as_float(s[124]), __uint_as_float(s[125]));
+                mx1 = fmax3(mx1, __uint_as_float(s[126]), __uint_as_float(s[127]));
                 const float mx_sc = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
+                if (row == 0) KSA_TR(1 + t, 3);
                 // lazy rescale: the reference max only moves when some row of the warp outgrew it
                 const bool need = mx_sc > m_used + kRescaleThreshold;
                 const bool need_any = __any_sync(0xffffffffu, need);
@@ -344,18 +385,21 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     l_run *= alpha;
                 }
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                const float2 sc2 = make_float2(scale_log2, scale_log2);
+                const float2 nm2 = make_float2(neg_m, neg_m);
+                float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+                // probabilities of the column pair (2q, 2q+1), packed into s[q]; the scale-and-shift
+                // and the row sum work on packed pairs (half the FMA-pipe instructions)
 #pragma unroll
-                for (int c = 0; c < 128; c += 4) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), scale_log2, neg_m));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), scale_log2, neg_m));
-                    const float p2 = ex2_approx(fmaf(__uint_as_float(s[c + 2]), scale_log2, neg_m));
-                    const float p3 = ex2_approx(fmaf(__uint_as_float(s[c + 3]), scale_log2, neg_m));
-                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                    s[c / 2] = pack_bf16x2(p0, p1);
-                    s[c / 2 + 1] = pack_bf16x2(p2, p3);
+                for (int q = 0; q < 64; ++q) {
+                    const float2 x = ffma2(make_float2(__uint_as_float(s[2 * q]), __uint_as_float(s[2 * q + 1])), sc2, nm2);
+                    float2 pr;
+                    pr.x = ex2_approx(x.x); pr.y = ex2_approx(x.y);
+                    if (q & 1) lb = fadd2(lb, pr); else la = fadd2(la, pr);
+                    s[q] = pack_bf16x2(pr.x, pr.y);
                 }
-                l_run += (l0 + l1) + (l2 + l3);
+                l_run += (la.x + la.y) + (lb.x + lb.y);
+                if (row == 0) KSA_TR(1 + t, 4);
                 {
                     uint32_t (&p0)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[0]);
                     uint32_t (&p1)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[32]);
@@ -375,7 +419,9 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_PFULL + t));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
+                if (row == 0) KSA_TR(1 + t, 6);
             }
             if (!alive) break;
             // ---- epilogue: O / l -> bf16 at the row's augmented position (Eq. 1), LSE ----
@@ -414,6 +460,17 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
     __syncthreads();
     if (warp == kProducerWarp) tmem_dealloc(tmem, 512);
 }
+
+#ifdef KSA_TRACE
+extern "C" __attribute__((visibility("default"))) int ksa_debug_read_trace(void* ev, void* cnt, int reset)
+{
+    cudaDeviceSynchronize();
+    if (ev) cudaMemcpyFromSymbol(ev, g_trace, sizeof(g_trace));
+    if (cnt) cudaMemcpyFromSymbol(cnt, g_trace_cnt, sizeof(g_trace_cnt));
+    if (reset) { static uint32_t z[8] = {0}; cudaMemcpyToSymbol(g_trace_cnt, z, sizeof(z)); }
+    return (int)cudaGetLastError();
+}
+#endif
 
 cudaError_t setup_text_tc()
 {
