@@ -39,8 +39,9 @@ using namespace ptx;
 // per role into a device buffer that ksa_debug_read_trace() copies out.  Compiled out by default.
 #ifdef KSA_TRACE
 constexpr int kTraceEvents = 8192;
-__device__ uint2 g_trace[2][4][kTraceEvents];
-__device__ uint32_t g_trace_cnt[2][4];
+constexpr int kTraceRoles = 12;             // 0 MMA issuer, 1-2 softmax row 0 of tile 0/1, 3 producer, 4-11 per-warp arrivals
+__device__ uint2 g_trace[2][kTraceRoles][kTraceEvents];
+__device__ uint32_t g_trace_cnt[2][kTraceRoles];
 #define KSA_TR(role, id)                                                                           \
     do {                                                                                           \
         if (tr_slot >= 0 && tr_n < (uint32_t)kTraceEvents) {                                       \
@@ -265,17 +266,21 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                         kstage = stage; kphase = ring_phase;
                         if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
                     }
+                    KSA_TR(0, 39);
                     if (!bounded_wait(kv_full(vstage), vphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                    KSA_TR(0, 40);
                     for (int t = 0; t < nh; ++t) {
                         if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
                         pf_phase[t] ^= 1u;
                         KSA_TR(0, 20 + t);
                         tc_fence_after();
                         issue_pv(t, vstage, j > 0);
+                        KSA_TR(0, 25 + t);
                         if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
                         if (j + 1 < T) {
                             if (t == 0) {
                                 if (!bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                                KSA_TR(0, 41);
                                 tc_fence_after();
                             }
                             issue_qk(t, kstage);
@@ -422,6 +427,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
                 if (row == 0) KSA_TR(1 + t, 6);
+                if (lane == 0 && row != 0) KSA_TR(4 + warp, 6);
             }
             if (!alive) break;
             // ---- epilogue: O / l -> bf16 at the row's augmented position (Eq. 1), LSE ----
@@ -467,7 +473,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_debug_read_trace(void*
     cudaDeviceSynchronize();
     if (ev) cudaMemcpyFromSymbol(ev, g_trace, sizeof(g_trace));
     if (cnt) cudaMemcpyFromSymbol(cnt, g_trace_cnt, sizeof(g_trace_cnt));
-    if (reset) { static uint32_t z[8] = {0}; cudaMemcpyToSymbol(g_trace_cnt, z, sizeof(z)); }
+    if (reset) { static uint32_t z[2 * kTraceRoles] = {0}; cudaMemcpyToSymbol(g_trace_cnt, z, sizeof(z)); }
     return (int)cudaGetLastError();
 }
 #endif
