@@ -144,42 +144,45 @@ __global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
     if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
 }
 
-// Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row):
-// one warp per (summary row, query head) as above, but every K and V row of the chunk is
-// requested before any is used (the loads overlap instead of forming a dependent chain), and
-// the per-key dot products are reduced across the warp together (independent shuffle chains).
+// Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row).
+// A block stages the K and V rows of kSummChunks consecutive chunks of one KV head in shared
+// memory (each row is read from global memory once, whatever the GQA group size), then its
+// warps take the (summary row, query head) tasks of those chunks: every key of the row is read
+// from shared memory before any is used, and the per-key dot products are reduced across the
+// warp together (independent shuffle chains).
 constexpr int kSummMaxKeys = 12;
+constexpr int kSummChunks = 8;
 
 template <int D>
 __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 {
     constexpr int E = D / 32;                     // dimensions per lane: 4 (8 bytes) or 2 (4 bytes)
     using Vec = typename std::conditional<E == 4, uint2, uint32_t>::type;
+    __shared__ __align__(16) uint16_t sK[kSummChunks * kSummMaxKeys * D];
+    __shared__ __align__(16) uint16_t sV[kSummChunks * kSummMaxKeys * D];
     const SeqInfo sq = a.seqs[blockIdx.y];
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int64_t total = (int64_t)sq.n_summ * a.Hq;
-    if (warp >= total) return;
-    const int u = (int)(warp / a.Hq);
-    const int h = (int)(warp - (int64_t)u * a.Hq);
-    const int hk = h / (a.Hq / a.Hkv);
-    const int j = u / a.m, r = u - j * a.m;
+    const int hk = blockIdx.z;
+    const int j0 = blockIdx.x * kSummChunks;
+    if (j0 >= sq.n_chunks) return;
+    const int nch = min(kSummChunks, sq.n_chunks - j0);
     const int s = a.k + a.m;
-    const int64_t key0 = sq.aug_off + (int64_t)j * s;
-    const int64_t qrow = key0 + a.k + r;
-    const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));
-
-    Vec kraw[kSummMaxKeys], vraw[kSummMaxKeys];
-    const Vec qraw = *reinterpret_cast<const Vec*>(a.q + qrow * a.q_st + (int64_t)h * a.q_sh + lane * E);
-#pragma unroll
-    for (int t = 0; t < kSummMaxKeys; ++t) {
-        if (t < nk) {
-            kraw[t] = *reinterpret_cast<const Vec*>(a.kx + (key0 + t) * a.k_st + (int64_t)hk * a.k_sh + lane * E);
-            vraw[t] = *reinterpret_cast<const Vec*>(a.v + (key0 + t) * a.v_st + (int64_t)hk * a.v_sh + lane * E);
-        } else {
-            kraw[t] = Vec(); vraw[t] = Vec();
+    const int G = a.Hq / a.Hkv;
+    const int64_t row0 = sq.aug_off + (int64_t)j0 * s;
+    // stage nch * s rows of K and V (16-byte vectors)
+    {
+        const int vecs = D / 8;
+        const int total = nch * s * vecs;
+        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+            const int rr = idx / vecs, vv = idx - rr * vecs;
+            const uint4 kx = *reinterpret_cast<const uint4*>(a.kx + (row0 + rr) * a.k_st + (int64_t)hk * a.k_sh + vv * 8);
+            const uint4 vx = *reinterpret_cast<const uint4*>(a.v + (row0 + rr) * a.v_st + (int64_t)hk * a.v_sh + vv * 8);
+            *reinterpret_cast<uint4*>(sK + rr * D + vv * 8) = kx;
+            *reinterpret_cast<uint4*>(sV + rr * D + vv * 8) = vx;
         }
     }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     auto unpack = [](const Vec& raw, float (&f)[E]) {
         const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw);
 #pragma unroll
@@ -188,47 +191,67 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
             f[e + 1] = __uint_as_float(w[e / 2] & 0xffff0000u);
         }
     };
-    float qv[E];
-    unpack(qraw, qv);
-    float x[kSummMaxKeys];
+    const int tasks = nch * a.m * G;
+    for (int task = wid; task < tasks; task += nwarps) {
+        const int g = task % G;
+        const int cr = task / G;
+        const int c = cr / a.m, r = cr - c * a.m;
+        const int h = hk * G + g;
+        const int64_t qrow = row0 + (int64_t)c * s + a.k + r;
+        const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));     // own-chunk text (+ own summaries 0..r)
+        const Vec qraw = *reinterpret_cast<const Vec*>(a.q + qrow * a.q_st + (int64_t)h * a.q_sh + lane * E);
+        const uint16_t* kbase = sK + c * s * D + lane * E;
+        const uint16_t* vbase = sV + c * s * D + lane * E;
+        float qv[E];
+        unpack(qraw, qv);
+        float x[kSummMaxKeys];
 #pragma unroll
-    for (int t = 0; t < kSummMaxKeys; ++t) {
-        float kf[E];
-        unpack(kraw[t], kf);
-        float dot = 0.f;
+        for (int t = 0; t < kSummMaxKeys; ++t) {
+            float dot = 0.f;
+            if (t < nk) {
+                float kf[E];
+                unpack(*reinterpret_cast<const Vec*>(kbase + t * D), kf);
 #pragma unroll
-        for (int e = 0; e < E; ++e) dot = fmaf(qv[e], kf[e], dot);
-        x[t] = dot;
+                for (int e = 0; e < E; ++e) dot = fmaf(qv[e], kf[e], dot);
+            }
+            x[t] = dot;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int t = 0; t < kSummMaxKeys; ++t)
+                if (t < s) x[t] += __shfl_xor_sync(0xffffffffu, x[t], o);
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int t = 0; t < kSummMaxKeys; ++t) {
+            x[t] = (t < nk) ? x[t] * a.scale : -INFINITY;
+            mx = fmaxf(mx, x[t]);
+        }
+        float l = 0.f, acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int t = 0; t < kSummMaxKeys; ++t) {
+            if (t < nk) {
+                const float p = __expf(x[t] - mx);
+                l += p;
+                float vf[E];
+                unpack(*reinterpret_cast<const Vec*>(vbase + t * D), vf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
+            }
+        }
+        const float inv = 1.f / l;
+        uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + lane * E;
+        Vec ov;
+        uint32_t* ow = reinterpret_cast<uint32_t*>(&ov);
+#pragma unroll
+        for (int e = 0; e < E; e += 2)
+            ow[e / 2] = (uint32_t)float_to_bf16_bits(acc[e] * inv) | ((uint32_t)float_to_bf16_bits(acc[e + 1] * inv) << 16);
+        *reinterpret_cast<Vec*>(op) = ov;
+        if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-        for (int t = 0; t < kSummMaxKeys; ++t)
-            if (t < s) x[t] += __shfl_xor_sync(0xffffffffu, x[t], o);
-    }
-    float mx = -INFINITY;
-#pragma unroll
-    for (int t = 0; t < kSummMaxKeys; ++t) {
-        x[t] = (t < nk) ? x[t] * a.scale : -INFINITY;
-        mx = fmaxf(mx, x[t]);
-    }
-    float l = 0.f, acc[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.f;
-#pragma unroll
-    for (int t = 0; t < kSummMaxKeys; ++t) {
-        const float p = __expf(x[t] - mx);                 // 0 for keys beyond nk
-        l += p;
-        float vf[E];
-        unpack(vraw[t], vf);
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
-    }
-    const float inv = 1.f / l;
-    uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
-    if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
 }
 
 cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
@@ -240,8 +263,10 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
     if (blocks < 1) blocks = 1;
     dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, 1);
     if (a.k + a.m <= kSummMaxKeys) {
-        if (a.D == 128) ksa_summary_short_kernel<128><<<grid, 256, 0, stream>>>(a);
-        else            ksa_summary_short_kernel<64><<<grid, 256, 0, stream>>>(a);
+        const int max_chunks = a.max_n_summ / a.m;
+        dim3 g2((unsigned)((max_chunks + kSummChunks - 1) / kSummChunks), (unsigned)a.num_seqs, (unsigned)a.Hkv);
+        if (a.D == 128) ksa_summary_short_kernel<128><<<g2, 256, 0, stream>>>(a);
+        else            ksa_summary_short_kernel<64><<<g2, 256, 0, stream>>>(a);
     } else {
         if (a.D == 128) ksa_summary_kernel<128><<<grid, 256, 0, stream>>>(a);
         else            ksa_summary_kernel<64><<<grid, 256, 0, stream>>>(a);
