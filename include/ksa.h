@@ -144,9 +144,15 @@ int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v,
 int ksa_host_staging_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
 /*
  * Same operator with HOST tensors (contiguous [total_aug, H, D]; strides in p are
- * ignored): copies q, k, v to the device staging buffer, runs ksa_attn_fwd, copies out
- * and lse back and synchronises the stream before returning.  Pinned host memory is
- * recommended.  staging: DEVICE, >= ksa_host_staging_bytes, 256-byte aligned.
+ * ignored).  The query tiles are cut into about eight row chunks in sequence order and
+ * pipelined: while one chunk's rows of q, k, v are copied to the device staging buffer
+ * (on a copy stream the context owns), the previous chunk is packed and computed on
+ * cuda_stream, and the one before that has its rows of out and lse copied back (on a
+ * second owned stream).  A chunk needs only keys at or before its own rows (Eq. 3), which
+ * earlier stages have uploaded.  Returns after both the last download and cuda_stream's
+ * work have completed.  Pinned host memory is needed for the copies to overlap.
+ * staging: DEVICE, >= ksa_host_staging_bytes, 256-byte aligned; scratch.
+ * The first call creates the two streams and a few events (kept until ksa_destroy).
  */
 int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                       void* out_host, float* lse_host, void* staging, size_t staging_bytes,

@@ -38,6 +38,10 @@ struct ksa_ctx {
     bool timing_valid = false;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     bool tc_ready = false;
+    // host entry point: copy streams and per-chunk events of its upload / compute / download pipeline
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_done;
+    cudaEvent_t ev_start = nullptr;
 };
 
 static int cuda_fail(ksa_ctx* ctx, cudaError_t e)
@@ -181,23 +185,56 @@ static BaseItem schedule_q_tile(const Eq3& e, const SeqInfo& s, int seq, int qt)
     return it;
 }
 
-void build_schedule(const ksa_params* p, HostSchedule& hs)
+void build_schedule(const ksa_params* p, HostSchedule& hs, int target_chunks)
 {
     const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
+    const int k = p->chunk_len, m = p->summaries_per_chunk, s = k + m;
     const int G = p->num_q_heads / p->num_kv_heads;
     const int heads_per_item = (G % 2 == 0) ? 2 : 1;
-    std::vector<BaseItem> base;
+    struct Tagged { BaseItem it; int32_t chunk; };
+    std::vector<Tagged> base;
+    hs.chunks.clear();
+    int64_t total_tiles = 0;
+    for (int b = 0; b < p->num_seqs; ++b) total_tiles += hs.seqs[b].text_pad / kTileM;
+    const int64_t per_chunk = target_chunks > 0 ? std::max<int64_t>(1, (total_tiles + target_chunks - 1) / target_chunks) : 0;
     for (int b = 0; b < p->num_seqs; ++b) {
-        const int n_qt = hs.seqs[b].text_pad / kTileM;
-        for (int qt = 0; qt < n_qt; ++qt) base.push_back(schedule_q_tile(e, hs.seqs[b], b, qt));
+        const SeqInfo& sq = hs.seqs[b];
+        const int n_qt = sq.text_pad / kTileM;
+        const int64_t n = sq.n_text, L = n + sq.n_summ;
+        auto aug_of = [&](int64_t i) -> int64_t { return i >= n ? L : (i / k) * s + (i % k); };   // Eq. 1
+        for (int qt = 0; qt < n_qt; ++qt) {
+            if (per_chunk > 0 && qt % per_chunk == 0) {
+                const int t0 = qt, t1 = (int)std::min<int64_t>(n_qt, qt + per_chunk);
+                const bool last = (t1 == n_qt);
+                const int64_t i0 = (int64_t)t0 * kTileM, i1 = last ? n : (int64_t)t1 * kTileM;
+                RowChunk c{};
+                c.seq = b;
+                c.text0 = (int32_t)i0; c.text1 = last ? sq.text_pad : (int32_t)i1;
+                // summaries of the full chunks whose rows end inside [i0, i1)
+                const int64_t j0 = i0 / k, j1 = last ? sq.n_chunks : i1 / k;
+                c.summ0 = (int32_t)(j0 * m); c.summq1 = (int32_t)(j1 * m);
+                c.summ1 = last ? sq.summ_pad : c.summq1;
+                c.aug0 = sq.aug_off + aug_of(i0); c.aug1 = sq.aug_off + aug_of(i1);
+                hs.chunks.push_back(c);
+            }
+            base.push_back({schedule_q_tile(e, sq, b, qt), (int32_t)hs.chunks.size() - 1});
+        }
     }
-    // longest first; ties keep (sequence, tile) order so that neighbours share K/V tiles in L2
-    std::stable_sort(base.begin(), base.end(), [](const BaseItem& x, const BaseItem& y) {
-        return (x.ns_tiles + x.band_hi - x.band_lo) > (y.ns_tiles + y.band_hi - y.band_lo);
+    // longest first (chunk by chunk, if chunked); ties keep (sequence, tile) order so that
+    // neighbours share K/V tiles in L2
+    std::stable_sort(base.begin(), base.end(), [](const Tagged& x, const Tagged& y) {
+        if (x.chunk != y.chunk) return x.chunk < y.chunk;
+        return (x.it.ns_tiles + x.it.band_hi - x.it.band_lo) > (y.it.ns_tiles + y.it.band_hi - y.it.band_lo);
     });
     hs.work.clear();
     hs.work.reserve(base.size() * (p->num_q_heads / heads_per_item));
-    for (const BaseItem& bi : base)
+    for (const Tagged& tg : base) {
+        const BaseItem& bi = tg.it;
+        if (tg.chunk >= 0) {
+            RowChunk& c = hs.chunks[tg.chunk];
+            if (c.work_cnt == 0) c.work_off = (int64_t)hs.work.size();
+            c.work_cnt += p->num_q_heads / heads_per_item;
+        }
         for (int h = 0; h < p->num_q_heads; h += heads_per_item) {
             WorkItem w{};
             w.seq = bi.seq; w.q_tile = bi.q_tile; w.head0 = h; w.n_heads = heads_per_item;
@@ -206,6 +243,7 @@ void build_schedule(const ksa_params* p, HostSchedule& hs)
             w.band_nomask_lo = bi.nm_lo; w.band_nomask_hi = bi.nm_hi;
             hs.work.push_back(w);
         }
+    }
 }
 
 static std::vector<int32_t> schedule_key(const ksa_params* p)
@@ -343,6 +381,11 @@ extern "C" __attribute__((visibility("default"))) int ksa_destroy(ksa_ctx* ctx)
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
     if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+    for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_done) cudaEventDestroy(e);
+    if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
+    if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
     delete ctx;
     return KSA_OK;
 }
@@ -384,14 +427,15 @@ extern "C" __attribute__((visibility("default"))) int ksa_text_kernel_ms(ksa_ctx
 // ---------------------------------------------------------------------------------------
 // schedule cache
 // ---------------------------------------------------------------------------------------
-static int ensure_schedule(ksa_ctx* ctx, const ksa_params* p, bool upload)
+static int ensure_schedule(ksa_ctx* ctx, const ksa_params* p, bool upload, int target_chunks = 0)
 {
     std::vector<int32_t> key = schedule_key(p);
+    key.push_back(target_chunks);
     if (ctx->sched.key != key) {
         HostSchedule hs;
         try {
             build_layout(p, hs);
-            build_schedule(p, hs);
+            build_schedule(p, hs, target_chunks);
         } catch (const std::bad_alloc&) { return KSA_ERR_NOMEM; }
         hs.key = key;
         ctx->sched = std::move(hs);
@@ -476,6 +520,60 @@ static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, 
     return KSA_OK;
 }
 
+// Kernel arguments of a whole problem (schedule already cached and uploaded in ctx).
+static KernelArgs make_args(ksa_ctx* ctx, const ksa_params* p, const void* q, const void* k, const void* v, void* out,
+                            float* lse, void* workspace, const WorkspaceLayout& wl)
+{
+    const HostSchedule& hs = ctx->sched;
+    char* ws = (char*)workspace;
+    KernelArgs a{};
+    a.seqs = ctx->d_seqs; a.work = ctx->d_work;
+    a.num_seqs = p->num_seqs; a.num_work = (int32_t)hs.work.size();
+    a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.C = p->window_chunks;
+    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.flags = p->flags;
+    a.scale = p->softmax_scale;
+    a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+    a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
+    a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
+    a.r_seq = -1;
+    a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v;
+    a.out = (uint16_t*)out; a.lse = lse;
+    a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;
+    a.v_st = p->v_stride_tok; a.v_sh = p->v_stride_head; a.o_st = p->o_stride_tok; a.o_sh = p->o_stride_head;
+    a.qt = (uint16_t*)(ws + wl.qt); a.kt = (uint16_t*)(ws + wl.kt); a.vt = (uint16_t*)(ws + wl.vt);
+    a.ks = (uint16_t*)(ws + wl.ks); a.vs = (uint16_t*)(ws + wl.vs);
+    a.status = ctx->d_status;
+    return a;
+}
+
+// One-time kernel setup and the tensor maps of the packed streams (tensor-core path only).
+static int prepare_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, TextMaps& maps)
+{
+    if (flags & KSA_FLAG_REFERENCE_KERNEL) return KSA_OK;
+    if (!ctx->tc_ready) {
+        cudaError_t e = setup_text_tc();
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->tc_ready = true;
+    }
+    int rc;
+    if ((rc = encode_stream_map(ctx, &maps.qt, a.qt, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
+    if ((rc = encode_stream_map(ctx, &maps.kt, a.kt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+    if ((rc = encode_stream_map(ctx, &maps.vt, a.vt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+    if ((rc = encode_stream_map(ctx, &maps.ks, a.ks, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+    return encode_stream_map(ctx, &maps.vs, a.vs, a.D, a.summ_rows, a.Hkv);
+}
+
+// Text-row kernel over the work items a.work[0 .. a.num_work).
+static int launch_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, const TextMaps& maps, cudaStream_t stream)
+{
+    cudaError_t e = (flags & KSA_FLAG_REFERENCE_KERNEL) ? launch_text_ref(a, stream)
+                                                        : launch_text_tc(a, maps, ctx->num_sms, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return KSA_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, void* out, float* lse,
                             void* workspace, size_t workspace_bytes, const ksa_params* p, void* cuda_stream)
 {
@@ -491,25 +589,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
     if (!workspace || workspace_bytes < wl.total || ((uintptr_t)workspace & 255)) return KSA_ERR_WORKSPACE;
 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    char* ws = (char*)workspace;
-    KernelArgs a{};
-    a.seqs = ctx->d_seqs; a.work = ctx->d_work;
-    a.num_seqs = p->num_seqs; a.num_work = (int32_t)hs.work.size();
-    a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.C = p->window_chunks;
-    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
-    a.flags = p->flags;
-    a.scale = p->softmax_scale;
-    a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
-    a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
-    a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
-    a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v;
-    a.out = (uint16_t*)out; a.lse = lse;
-    a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;
-    a.v_st = p->v_stride_tok; a.v_sh = p->v_stride_head; a.o_st = p->o_stride_tok; a.o_sh = p->o_stride_head;
-    a.qt = (uint16_t*)(ws + wl.qt); a.kt = (uint16_t*)(ws + wl.kt); a.vt = (uint16_t*)(ws + wl.vt);
-    a.ks = (uint16_t*)(ws + wl.ks); a.vs = (uint16_t*)(ws + wl.vs);
-    a.status = ctx->d_status;
-
+    KernelArgs a = make_args(ctx, p, q, k, v, out, lse, workspace, wl);
     cudaError_t e;
     if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
@@ -518,25 +598,15 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
         ctx->launches += 1;
     }
     if (ctx->timing) cudaEventRecord(ctx->ev0, stream);
-    if (p->flags & KSA_FLAG_REFERENCE_KERNEL) {
-        if ((e = launch_text_ref(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    } else {
-        if (!ctx->tc_ready) {
-            if ((e = setup_text_tc()) != cudaSuccess) return cuda_fail(ctx, e);
-            ctx->tc_ready = true;
-        }
-        TextMaps maps;
-        if ((rc = encode_stream_map(ctx, &maps.qt, a.qt, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &maps.kt, a.kt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &maps.vt, a.vt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &maps.ks, a.ks, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &maps.vs, a.vs, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((e = launch_text_tc(a, maps, ctx->num_sms, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    }
-    ctx->launches += 1;
+    TextMaps maps;
+    if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
+    if ((rc = launch_text(ctx, a, p->flags, maps, stream)) != KSA_OK) return rc;
     if (ctx->timing) { cudaEventRecord(ctx->ev1, stream); ctx->timing_valid = true; }
     return KSA_OK;
 }
+
+// Number of row chunks the host entry point aims for (upload / compute / download stages).
+static constexpr int kHostPipelineChunks = 8;
 
 struct StagingLayout { size_t q, k, v, out, lse, ws, ws_bytes, total; };
 static int staging_layout(const ksa_params* p, StagingLayout& s)
@@ -581,21 +651,85 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_host(ksa_ctx*
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* d = (char*)staging;
     const size_t D2 = (size_t)p->head_dim * 2;
-    const int64_t total_aug = ksa_total_aug_len(p);
-    const size_t qb = (size_t)total_aug * p->num_q_heads * D2, kb = (size_t)total_aug * p->num_kv_heads * D2;
-    const size_t lb = (size_t)total_aug * p->num_q_heads * 4;
-    cudaError_t e;
-    if ((e = cudaMemcpyAsync(d + s.q, q_host, qb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = cudaMemcpyAsync(d + s.k, k_host, kb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = cudaMemcpyAsync(d + s.v, v_host, kb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     ksa_params pc = *p;   // contiguous device images
     pc.q_stride_tok = pc.o_stride_tok = (int64_t)p->num_q_heads * p->head_dim;
     pc.k_stride_tok = pc.v_stride_tok = (int64_t)p->num_kv_heads * p->head_dim;
     pc.q_stride_head = pc.k_stride_head = pc.v_stride_head = pc.o_stride_head = p->head_dim;
-    rc = ksa_attn_fwd(ctx, d + s.q, d + s.k, d + s.v, d + s.out, (float*)(d + s.lse), d + s.ws, s.ws_bytes, &pc, stream);
-    if (rc != KSA_OK) return rc;
-    if ((e = cudaMemcpyAsync(out_host, d + s.out, qb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = cudaMemcpyAsync(lse_host, d + s.lse, lb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+
+    // Upload, compute and download overlap: the query tiles are cut into row chunks in sequence
+    // order.  A chunk's rows of q, k, v are contiguous on the host; its text rows only need keys at
+    // or before their own position (Eq. 3) and its summary rows only their own chunk, all of which
+    // earlier stages have already uploaded and packed; its rows of out are contiguous too.
+    // Stage c: copy-in stream uploads chunk c -> caller's stream packs it, runs its summary rows and
+    // its share of the work list -> copy-out stream downloads its out / lse rows.
+    if ((rc = ensure_schedule(ctx, &pc, true, kHostPipelineChunks)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    const WorkspaceLayout wl = workspace_layout(&pc, hs);
+    cudaError_t e;
+    if (!ctx->s_in) {
+        if ((e = cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(ctx, e);
+        if ((e = cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(ctx, e);
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    while (ctx->ev_in.size() < hs.chunks.size()) {
+        cudaEvent_t a0, a1;
+        if ((e = cudaEventCreateWithFlags(&a0, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(ctx, e);
+        if ((e = cudaEventCreateWithFlags(&a1, cudaEventDisableTiming)) != cudaSuccess) { cudaEventDestroy(a0); return cuda_fail(ctx, e); }
+        ctx->ev_in.push_back(a0); ctx->ev_done.push_back(a1);
+    }
+    KernelArgs a = make_args(ctx, &pc, d + s.q, d + s.k, d + s.v, d + s.out, (float*)(d + s.lse), d + s.ws, wl);
+    TextMaps maps;
+    if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
+    // the copy-in stream starts after whatever the caller queued before this call
+    if ((e = cudaEventRecord(ctx->ev_start, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamWaitEvent(ctx->s_in, ctx->ev_start, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+    const size_t q_row = (size_t)p->num_q_heads * D2, kv_row = (size_t)p->num_kv_heads * D2;
+    const WorkItem* work_base = a.work;
+    for (size_t ci = 0; ci < hs.chunks.size(); ++ci) {
+        const RowChunk& c = hs.chunks[ci];
+        const size_t r0 = (size_t)c.aug0, nr = (size_t)(c.aug1 - c.aug0);
+        if (nr > 0) {
+            if ((e = cudaMemcpyAsync(d + s.q + r0 * q_row, (const char*)q_host + r0 * q_row, nr * q_row, cudaMemcpyHostToDevice, ctx->s_in)) != cudaSuccess) return cuda_fail(ctx, e);
+            if ((e = cudaMemcpyAsync(d + s.k + r0 * kv_row, (const char*)k_host + r0 * kv_row, nr * kv_row, cudaMemcpyHostToDevice, ctx->s_in)) != cudaSuccess) return cuda_fail(ctx, e);
+            if ((e = cudaMemcpyAsync(d + s.v + r0 * kv_row, (const char*)v_host + r0 * kv_row, nr * kv_row, cudaMemcpyHostToDevice, ctx->s_in)) != cudaSuccess) return cuda_fail(ctx, e);
+        }
+        if ((e = cudaEventRecord(ctx->ev_in[ci], ctx->s_in)) != cudaSuccess) return cuda_fail(ctx, e);
+        if ((e = cudaStreamWaitEvent(stream, ctx->ev_in[ci], 0)) != cudaSuccess) return cuda_fail(ctx, e);
+        a.r_seq = c.seq;
+        a.r_text0 = c.text0; a.r_text1 = c.text1;
+        a.r_summ0 = c.summ0; a.r_summ1 = c.summ1; a.r_summq1 = c.summq1;
+        if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+        // The last summary tile this stage's text rows visit may reach past the rows packed so far
+        // (those belong to later stages and are masked out).  Their V rows must still be finite,
+        // or 0 * V would poison the accumulators: clear them up to the tile boundary.
+        {
+            const SeqInfo& sq = hs.seqs[c.seq];
+            const int64_t z0 = c.summ1, z1 = std::min<int64_t>(sq.summ_pad, round_up(c.summ1, kTileN));
+            if (z1 > z0) {
+                char* vs_rows = (char*)a.vs + ((size_t)sq.summ_off + (size_t)z0) * D2;
+                if ((e = cudaMemset2DAsync(vs_rows, (size_t)hs.summ_rows * D2, 0, (size_t)(z1 - z0) * D2, (size_t)p->num_kv_heads,
+                                           stream)) != cudaSuccess) return cuda_fail(ctx, e);
+            }
+        }
+        if (a.m > 0 && c.summq1 > c.summ0) {
+            if ((e = launch_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+            ctx->launches += 1;
+        }
+        a.work = work_base + c.work_off;
+        a.num_work = (int32_t)c.work_cnt;
+        if ((rc = launch_text(ctx, a, p->flags, maps, stream)) != KSA_OK) return rc;
+        if ((e = cudaEventRecord(ctx->ev_done[ci], stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        if ((e = cudaStreamWaitEvent(ctx->s_out, ctx->ev_done[ci], 0)) != cudaSuccess) return cuda_fail(ctx, e);
+        if (nr > 0) {
+            if ((e = cudaMemcpyAsync((char*)out_host + r0 * q_row, d + s.out + r0 * q_row, nr * q_row, cudaMemcpyDeviceToHost, ctx->s_out)) != cudaSuccess) return cuda_fail(ctx, e);
+            // lse is [heads, total rows]: one strip of nr columns per head
+            const size_t pitch = (size_t)hs.total_aug * 4;
+            if ((e = cudaMemcpy2DAsync((char*)lse_host + r0 * 4, pitch, d + s.lse + r0 * 4, pitch, nr * 4, (size_t)p->num_q_heads,
+                                       cudaMemcpyDeviceToHost, ctx->s_out)) != cudaSuccess) return cuda_fail(ctx, e);
+        }
+    }
+    if ((e = cudaStreamSynchronize(ctx->s_out)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(ctx, e);
     return KSA_OK;
 }

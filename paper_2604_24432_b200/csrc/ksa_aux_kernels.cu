@@ -24,19 +24,22 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) ksa_pack_kernel(KernelArgs a)
 {
-    const SeqInfo sq = a.seqs[blockIdx.y];
+    const bool ranged = a.r_seq >= 0;
+    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const bool text = (blockIdx.z == 0);
     const int vecs = a.D / 8;
     const int slots = text ? (a.Hq + 2 * a.Hkv) : (2 * a.Hkv);
-    const int pad_rows = text ? sq.text_pad : sq.summ_pad;
+    const int row_first = ranged ? (text ? a.r_text0 : a.r_summ0) : 0;
+    const int pad_rows = (ranged ? (text ? a.r_text1 : a.r_summ1) : (text ? sq.text_pad : sq.summ_pad)) - row_first;
     const int live_rows = text ? sq.n_text : sq.n_summ;
     const int64_t per_row = (int64_t)slots * vecs;
     const int64_t total = (int64_t)pad_rows * per_row;
     const int s = a.k + a.m;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (int64_t)gridDim.x * blockDim.x) {
-        const int row = (int)(idx / per_row);
-        const int rem = (int)(idx - (int64_t)row * per_row);
+        const int row_rel = (int)(idx / per_row);
+        const int rem = (int)(idx - (int64_t)row_rel * per_row);
+        const int row = row_first + row_rel;
         const int slot = rem / vecs;
         const int vec = rem - slot * vecs;
         int64_t aug = 0;
@@ -81,11 +84,12 @@ cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream)
 {
     // grid.x covers the longest padded stream of any sequence (grid-stride loop beyond the cap).
     const int64_t per_row = (int64_t)(a.Hq + 2 * a.Hkv) * (a.D / 8);
-    const int64_t rows = a.max_text_pad > a.max_summ_pad ? a.max_text_pad : a.max_summ_pad;
+    int64_t rows = a.max_text_pad > a.max_summ_pad ? a.max_text_pad : a.max_summ_pad;
+    if (a.r_seq >= 0) rows = (a.r_text1 - a.r_text0) > (a.r_summ1 - a.r_summ0) ? (a.r_text1 - a.r_text0) : (a.r_summ1 - a.r_summ0);
     int64_t blocks = (rows * per_row + 255) / 256;
     if (blocks > 148 * 64) blocks = 148 * 64;
     if (blocks < 1) blocks = 1;
-    dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, a.m > 0 ? 2u : 1u);
+    dim3 grid((unsigned)blocks, a.r_seq >= 0 ? 1u : (unsigned)a.num_seqs, a.m > 0 ? 2u : 1u);
     ksa_pack_kernel<<<grid, 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
@@ -99,13 +103,15 @@ template <int D>
 __global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
 {
     constexpr int E = D / 32;
-    const SeqInfo sq = a.seqs[blockIdx.y];
+    const bool ranged = a.r_seq >= 0;
+    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int64_t total = (int64_t)sq.n_summ * a.Hq;
+    const int u_first = ranged ? a.r_summ0 : 0;
+    const int64_t total = (int64_t)((ranged ? a.r_summq1 : sq.n_summ) - u_first) * a.Hq;
     if (warp >= total) return;
-    const int u = (int)(warp / a.Hq);
-    const int h = (int)(warp - (int64_t)u * a.Hq);
+    const int u = u_first + (int)(warp / a.Hq);
+    const int h = (int)(warp % a.Hq);
     const int hk = h / (a.Hq / a.Hkv);
     const int j = u / a.m, r = u - j * a.m;
     const int s = a.k + a.m;
@@ -160,11 +166,15 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
     using Vec = typename std::conditional<E == 4, uint2, uint32_t>::type;
     __shared__ __align__(16) uint16_t sK[kSummChunks * kSummMaxKeys * D];
     __shared__ __align__(16) uint16_t sV[kSummChunks * kSummMaxKeys * D];
-    const SeqInfo sq = a.seqs[blockIdx.y];
+    const bool ranged = a.r_seq >= 0;
+    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const int hk = blockIdx.z;
-    const int j0 = blockIdx.x * kSummChunks;
-    if (j0 >= sq.n_chunks) return;
-    const int nch = min(kSummChunks, sq.n_chunks - j0);
+    // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
+    const int j_first = ranged ? a.r_summ0 / a.m : 0;
+    const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
+    const int j0 = j_first + blockIdx.x * kSummChunks;
+    if (j0 >= j_end) return;
+    const int nch = min(kSummChunks, j_end - j0);
     const int s = a.k + a.m;
     const int G = a.Hq / a.Hkv;
     const int64_t row0 = sq.aug_off + (int64_t)j0 * s;
@@ -258,13 +268,16 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
 {
     if (a.m <= 0 || a.max_n_summ <= 0) return cudaSuccess;
     // grid.x covers the sequence with the most summary rows; shorter ones exit early.
-    const int64_t warps = (int64_t)a.max_n_summ * a.Hq;
+    const int rows = a.r_seq >= 0 ? (a.r_summq1 - a.r_summ0) : a.max_n_summ;
+    if (rows <= 0) return cudaSuccess;
+    const unsigned ny = a.r_seq >= 0 ? 1u : (unsigned)a.num_seqs;
+    const int64_t warps = (int64_t)rows * a.Hq;
     int64_t blocks = (warps + 7) / 8;
     if (blocks < 1) blocks = 1;
-    dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, 1);
+    dim3 grid((unsigned)blocks, ny, 1);
     if (a.k + a.m <= kSummMaxKeys) {
-        const int max_chunks = a.max_n_summ / a.m;
-        dim3 g2((unsigned)((max_chunks + kSummChunks - 1) / kSummChunks), (unsigned)a.num_seqs, (unsigned)a.Hkv);
+        const int max_chunks = rows / a.m;
+        dim3 g2((unsigned)((max_chunks + kSummChunks - 1) / kSummChunks), ny, (unsigned)a.Hkv);
         if (a.D == 128) ksa_summary_short_kernel<128><<<g2, 256, 0, stream>>>(a);
         else            ksa_summary_short_kernel<64><<<g2, 256, 0, stream>>>(a);
     } else {

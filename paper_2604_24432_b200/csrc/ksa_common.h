@@ -53,7 +53,11 @@ struct KernelArgs {
     int32_t max_text_pad;   // largest per-sequence padded text rows
     int32_t max_summ_pad;   // largest per-sequence padded summary rows
     int32_t max_n_summ;     // largest per-sequence summary count
-    int32_t reserved;
+    // Row range (pack and summary kernels): r_seq < 0 means every sequence in full; otherwise only
+    // sequence r_seq, packed text rows [r_text0, r_text1), summary-stream rows [r_summ0, r_summ1)
+    // (pack) and summary query rows [r_summ0, r_summq1) (summary-row kernel).
+    int32_t r_seq;
+    int32_t r_text0, r_text1, r_summ0, r_summ1, r_summq1;
     // user tensors (bf16 as uint16)
     const uint16_t* q; const uint16_t* kx; const uint16_t* v; uint16_t* out; float* lse;
     int64_t q_st, q_sh, k_st, k_sh, v_st, v_sh, o_st, o_sh;

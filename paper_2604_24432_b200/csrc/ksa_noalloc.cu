@@ -138,6 +138,7 @@ int ksa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
     a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
     a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
     a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
+    a.r_seq = -1;
     a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v;
     a.out = (uint16_t*)out; a.lse = lse;
     a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;

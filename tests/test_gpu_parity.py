@@ -103,17 +103,29 @@ def test_strided_inputs_and_stream(ctx):
     assert (outbuf[:, 0] == 0).all()
 
 
-def test_host_entry_point(ctx):
-    wl = synth.Workload("host", 6, [500, 300], 4, 2, 128)
-    total = orc.aug_len(500, 8, 1) + orc.aug_len(300, 8, 1)
-    q, k, v = synth.make_qkv(wl, total, pin=True)
-    prob = ksa.Problem([500, 300], 8, 1, 2, 4, 2, 128, wl.scale)
-    out = torch.empty((total, 4, 128), dtype=torch.bfloat16).pin_memory()
-    lse = torch.empty((4, total), dtype=torch.float32).pin_memory()
-    staging = torch.empty(ksa.host_staging_bytes(prob), dtype=torch.uint8, device="cuda:0")
-    ctx.attn_fwd_host(prob, q, k, v, out, lse, staging)
-    ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), [500, 300], 8, 1, 2, wl.scale)
-    parity.compare(out.double().numpy(), lse.double().numpy().T, ref_out, ref_lse, "host")
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv", [
+    ([500, 300], 8, 1, 2, 4, 2),          # shorter than a row chunk each
+    ([6000], 8, 1, 16, 8, 2),             # one sequence cut into several upload/compute/download stages
+    ([5000, 1300, 77], 3, 2, 5, 6, 2),    # k does not divide the tile, m = 2, ragged lengths, G = 3
+    ([3000, 2100], 16, 0, 7, 4, 4),       # no summaries
+])
+def test_host_entry_point(ctx, lens, k, m, C, Hq, Hkv):
+    """Host tensors in, host tensors out (the pipelined entry point).  The staging buffer starts
+    out filled with NaN bit patterns: nothing that a stage has not written yet may leak into a result."""
+    wl = synth.Workload("host", 6, lens, Hq, Hkv, 128)
+    total = sum(orc.aug_len(n, k, m) for n in lens)
+    q, kk, v = synth.make_qkv(wl, total, pin=True)
+    prob = ksa.Problem(lens, k, m, C, Hq, Hkv, 128, wl.scale)
+    out = torch.empty((total, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    lse = torch.empty((Hq, total), dtype=torch.float32).pin_memory()
+    staging = torch.full((ksa.host_staging_bytes(prob),), 0xFF, dtype=torch.uint8, device="cuda:0")
+    for _ in range(2):                    # the second call reuses the cached chunked schedule
+        out.fill_(7.0); lse.fill_(-1.0)
+        ctx.clear_device_status()
+        ctx.attn_fwd_host(prob, q, kk, v, out, lse, staging)
+        assert ctx.device_status() == 0
+        ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(kk), synth.bits(v), lens, k, m, C, wl.scale)
+        parity.compare(out.double().numpy(), lse.double().numpy().T, ref_out, ref_lse, "host")
 
 
 def test_runtime_argument_errors(ctx):
