@@ -31,6 +31,8 @@ EXPORTS = [
     "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
     "ksa_last_cuda_error", "ksa_launch_count", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
     "ksa_strerror",
+    "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
+    "ksa_decode_text", "ksa_decode_summary",
 ]
 
 
@@ -47,6 +49,15 @@ class ksa_params(ctypes.Structure):
         ("v_stride_tok", ctypes.c_int64), ("v_stride_head", ctypes.c_int64),
         ("o_stride_tok", ctypes.c_int64), ("o_stride_head", ctypes.c_int64),
         ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+    ]
+
+
+class ksa_cache_params(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_int32), ("batch", ctypes.c_int32), ("chunk_len", ctypes.c_int32),
+        ("window_chunks", ctypes.c_int32), ("max_summaries", ctypes.c_int32),
+        ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
     ]
 
 
@@ -96,6 +107,16 @@ def lib():
     L.ksa_launch_count.argtypes = [vp]
     L.ksa_enable_kernel_timing.argtypes = [vp, ctypes.c_int]
     L.ksa_text_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    cp = ctypes.POINTER(ksa_cache_params)
+    szp = ctypes.POINTER(ctypes.c_size_t)
+    L.ksa_cache_rows.restype = i64
+    L.ksa_cache_rows.argtypes = [cp]
+    L.ksa_cache_bytes.argtypes = [cp, szp, szp, szp]
+    L.ksa_cache_slice.argtypes = [cp, i64, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    L.ksa_cache_reset.argtypes = [vp, vp, cp, vp]
+    L.ksa_cache_fill_from_prefill.argtypes = [vp, vp, vp, vp, vp, vp, pp, cp, vp]
+    L.ksa_decode_text.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, cp, vp]
+    L.ksa_decode_summary.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, cp, vp]
     L.ksa_strerror.restype = ctypes.c_char_p
     L.ksa_strerror.argtypes = [ctypes.c_int]
     _lib = L
@@ -283,3 +304,88 @@ def attn_fwd(ctx: Context, prob: Problem, q, k, v):
     ws = torch.empty(workspace_bytes(prob), dtype=torch.uint8, device=q.device)
     ctx.attn_fwd(prob, q, k, v, out, lse, ws)
     return out, lse
+
+
+@dataclass
+class CacheSpec:
+    """Python-side holder of a ``ksa_cache_params`` (decode path, Sec. 2.3.1)."""
+    batch: int
+    k: int
+    C: int
+    max_summaries: int
+    Hq: int
+    Hkv: int
+    D: int
+    scale: float
+    flags: int = 0
+
+    def params(self) -> ksa_cache_params:
+        p = ksa_cache_params()
+        p.struct_size = ctypes.sizeof(ksa_cache_params)
+        p.batch, p.chunk_len, p.window_chunks, p.max_summaries = self.batch, self.k, self.C, self.max_summaries
+        p.num_q_heads, p.num_kv_heads, p.head_dim = self.Hq, self.Hkv, self.D
+        p.softmax_scale, p.flags = self.scale, self.flags
+        return p
+
+
+def cache_rows(spec: CacheSpec) -> int:
+    p = spec.params()
+    return int(lib().ksa_cache_rows(ctypes.byref(p)))
+
+
+def cache_bytes(spec: CacheSpec):
+    """(bytes of kcache = vcache, bytes of the state array, bytes of the decode workspace)"""
+    p = spec.params()
+    a, b, c = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().ksa_cache_bytes(ctypes.byref(p), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "ksa_cache_bytes")
+    return int(a.value), int(b.value), int(c.value)
+
+
+def cache_slice(spec: CacheSpec, text_tokens_before: int, is_summary: bool):
+    p = spec.params()
+    lo, hi = ctypes.c_int64(), ctypes.c_int64()
+    _check(lib().ksa_cache_slice(ctypes.byref(p), text_tokens_before, int(is_summary), ctypes.byref(lo), ctypes.byref(hi)),
+           "ksa_cache_slice")
+    return int(lo.value), int(hi.value)
+
+
+class DecodeCache:
+    """Torch tensors of one Summary KV cache plus the calls that step it (argument marshalling only)."""
+
+    def __init__(self, ctx: "Context", spec: CacheSpec):
+        import torch
+        self.ctx, self.spec = ctx, spec
+        dev = torch.device("cuda", ctx.device)
+        rows = cache_rows(spec)
+        _, _, wsb = cache_bytes(spec)
+        self.kcache = torch.zeros((spec.batch, spec.Hkv, rows, spec.D), dtype=torch.bfloat16, device=dev)
+        self.vcache = torch.zeros_like(self.kcache)
+        self.state = torch.zeros((spec.batch, 2), dtype=torch.int32, device=dev)
+        self.workspace = torch.empty(max(wsb, 256), dtype=torch.uint8, device=dev)
+
+    def _stream(self, stream):
+        import torch
+        return torch.cuda.current_stream(self.kcache.device).cuda_stream if stream is None else stream
+
+    def reset(self, stream=None):
+        p = self.spec.params()
+        _check(lib().ksa_cache_reset(self.ctx.handle, self.state.data_ptr(), ctypes.byref(p), self._stream(stream)), "ksa_cache_reset")
+
+    def fill_from_prefill(self, prob: Problem, k, v, stream=None):
+        p = self.spec.params()
+        pp_ = prob.params(None, k, v, None)
+        _check(lib().ksa_cache_fill_from_prefill(self.ctx.handle, self.kcache.data_ptr(), self.vcache.data_ptr(), self.state.data_ptr(),
+                                                 k.data_ptr(), v.data_ptr(), ctypes.byref(pp_), ctypes.byref(p), self._stream(stream)),
+               "ksa_cache_fill_from_prefill")
+
+    def _step(self, fn, name, q, k_new, v_new, out, lse, stream):
+        p = self.spec.params()
+        _check(fn(self.ctx.handle, self.kcache.data_ptr(), self.vcache.data_ptr(), self.state.data_ptr(), q.data_ptr(),
+                  k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), lse.data_ptr(), self.workspace.data_ptr(),
+                  self.workspace.numel(), ctypes.byref(p), self._stream(stream)), name)
+
+    def decode_text(self, q, k_new, v_new, out, lse, stream=None):
+        self._step(lib().ksa_decode_text, "ksa_decode_text", q, k_new, v_new, out, lse, stream)
+
+    def decode_summary(self, q, k_new, v_new, out, lse, stream=None):
+        self._step(lib().ksa_decode_summary, "ksa_decode_summary", q, k_new, v_new, out, lse, stream)

@@ -50,6 +50,11 @@ static int cuda_fail(ksa_ctx* ctx, cudaError_t e)
     return KSA_ERR_CUDA;
 }
 
+int32_t* ksa_ctx_status_word(ksa_ctx* ctx) { return ctx->d_status; }
+int ksa_ctx_num_sms(const ksa_ctx* ctx) { return ctx->num_sms; }
+void ksa_ctx_add_launches(ksa_ctx* ctx, int n) { ctx->launches += n; }
+int ksa_ctx_cuda_fail(ksa_ctx* ctx, int cuda_error) { return cuda_fail(ctx, (cudaError_t)cuda_error); }
+
 // ---------------------------------------------------------------------------------------
 // validation and layout
 // ---------------------------------------------------------------------------------------

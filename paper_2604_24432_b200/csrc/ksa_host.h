@@ -38,3 +38,9 @@ void build_layout(const ksa_params* p, HostSchedule& hs);
 void build_schedule(const ksa_params* p, HostSchedule& hs, int target_chunks = 0);
 // Offsets of the packed streams inside the workspace, and its total size.
 WorkspaceLayout workspace_layout(const ksa_params* p, const HostSchedule& hs);
+
+// Access to the context for the other entry-point files (the struct itself lives in ksa_api.cu).
+int32_t* ksa_ctx_status_word(ksa_ctx* ctx);                 // device status word
+int ksa_ctx_num_sms(const ksa_ctx* ctx);
+void ksa_ctx_add_launches(ksa_ctx* ctx, int n);
+int ksa_ctx_cuda_fail(ksa_ctx* ctx, int cuda_error);        // records the error, returns KSA_ERR_CUDA
