@@ -311,6 +311,87 @@ def run_ours(args):
     return 0
 
 
+# ---------------------------------------------------------------------------------------
+# decode path (secondary line): one auto-regressive step over the Summary KV cache
+# ---------------------------------------------------------------------------------------
+def run_decode(args):
+    """python bench.py --decode: B sequences at a 128K-token context (layout P, GQA 32/4, D 128), each step
+    appends one text token per sequence and attends over the cache slice; every k-th step is followed by
+    the chunk's summary step.  HBM-bound: the roofline is the measured copy bandwidth."""
+    from paper_2604_24432_b200 import binding as ksa
+    from paper_2604_24432_b200 import build as ksa_build
+    rank, world, local = dist_env()
+    if rank != 0:
+        return 0
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ksa_build.build()
+    B, k, C, Hq, Hkv, D = args.decode_batch, 8, 128, 32, 4, 128
+    ctx_len = 131072
+    steps, warm = args.steps, max(args.warmup, 3)
+    spec = ksa.CacheSpec(B, k, C, ctx_len // k + (steps + warm) // k + 2, Hq, Hkv, D, float(np.float32(1.0 / np.sqrt(D))))
+    ctx = ksa.Context(local)
+    cache = ksa.DecodeCache(ctx, spec)
+    g = torch.Generator(device=dev).manual_seed(5)
+    cache.kcache.normal_(generator=g); cache.vcache.normal_(generator=g)
+    pos0 = ctx_len - k * ((warm + k - 1) // k)          # chunk-aligned start so that the timed region starts at ctx_len
+    cache.state[:, 0] = pos0; cache.state[:, 1] = pos0 // k
+    q = torch.randn((B, Hq, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    kn = torch.randn((B, Hkv, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    vn = torch.randn((B, Hkv, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step(pos):
+        cache.decode_text(q, kn, vn, out, lse)
+        if (pos + 1) % k == 0:
+            cache.decode_summary(q, kn, vn, out, lse)
+        return pos + 1
+
+    pos = pos0
+    while pos < ctx_len:
+        pos = step(pos)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    launches0 = ctx.launch_count()
+    bytes_read = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record(stream)
+        for _ in range(steps):
+            lo, hi = ksa.cache_slice(spec, pos, False)
+            bytes_read += B * Hkv * (hi - lo) * D * 2 * 2
+            if (pos + 1) % k == 0:
+                bytes_read += B * Hkv * (k + 1) * D * 2 * 2
+            pos = step(pos)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert ctx.device_status() == 0
+    st = cache.state.cpu().numpy()
+    assert (st[:, 0] == pos).all() and (st[:, 1] == pos // k).all()
+    peaks = load_peaks()
+    gbs = bytes_read / steps / (ms * 1e-3) / 1e9
+    cache_gb = 2 * cache.kcache.numel() * 2 / 1e9
+    line = {
+        "metric": "KSA decode step over the Summary KV cache: tokens/s at a 128K context", "value": B / (ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)",
+        "config": {"workload": f"decode, {B} sequences at {ctx_len} cached text tokens each", "layout": f"P: k={k} m=1 C={C}",
+                   "heads": f"{Hq}q/{Hkv}kv", "head_dim": D, "cache_gb": cache_gb,
+                   "l2_policy": "the cache slices read per step are larger than L2 (no flush)", "parallelism": "1 GPU"},
+        "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": f"of {peaks['source']} (copy bandwidth)",
+                     "kernel": "ksa_decode_attn_kernel (+ append, merge, commit)",
+                     "bytes_per_step": bytes_read / steps},
+        "e2e": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def summary_pairs(wl, layout):
     """Visible pairs of the summary rows (they run in their own small kernel)."""
     tot = 0
@@ -332,9 +413,13 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
+    ap.add_argument("--decode-batch", type=int, default=32)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.decode:
+        return run_decode(args)
     return run_ours(args)
 
 
