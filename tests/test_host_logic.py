@@ -22,15 +22,19 @@ def _built():
 
 
 def test_exports_match_header():
-    hdr = open(os.path.join(ROOT, "include", "ksa.h")).read()
-    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    declared = set(re.findall(r"\b(ksa_[a-z_]+)\s*\(", hdr))
+    declared = set()
+    inc = os.path.join(ROOT, "include")
+    for name in sorted(os.listdir(inc)):            # every header of the C ABI
+        hdr = open(os.path.join(inc, name)).read()
+        hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+        declared |= set(re.findall(r"\b(ksa_[a-z_]+)\s*\(", hdr))
     assert declared == set(ksa.EXPORTS)
     L = ksa.lib()
     for name in declared:
         assert hasattr(L, name), name
     assert ctypes.sizeof(ksa.ksa_params) == 120
     assert ctypes.sizeof(ksa.ksa_tile_rec) == 32
+    assert ctypes.sizeof(ksa.ksa_cache_params) == 40
 
 
 def test_aug_len_and_pairs_match_oracle():
