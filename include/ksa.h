@@ -127,10 +127,18 @@ int ksa_visible_pairs(const ksa_params* p, int64_t* pairs);
  *   out       DEVICE bf16, same shape as q (strides o_stride_*); every row is written
  *   lse       DEVICE fp32 [num_q_heads, total_aug]; every entry is written
  *   workspace DEVICE, >= ksa_workspace_bytes, 256-byte aligned; contents are scratch and
- *             must not be used by other work on other streams while the call runs
+ *             must not be used by other work on other streams while the call runs.  When
+ *             every sequence is a whole number of chunks (the paper's assumption) and a
+ *             128-row tile is a whole number of chunks (128 % k == 0, 128 % m == 0 or
+ *             m == 0), ksa_workspace_bytes is 256 and the workspace is not touched: the
+ *             text-row kernel reads its tiles straight from q, k, v through chunked
+ *             4-D tensor maps and nothing is packed
  *   cuda_stream  a cudaStream_t (NULL = legacy default stream)
- * Steps enqueued: pack (de-interleave text Q/K/V and summary K/V into dense streams),
- * summary-row attention, text-row attention over the scheduled tiles.
+ * Steps enqueued: pack (de-interleave text Q/K/V and summary K/V into dense streams;
+ * skipped in the case above), summary-row attention, text-row attention over the
+ * scheduled tiles.  In the no-pack case the padding rows of a partial tile hold rows
+ * of the following sequence; they are masked, but like any masked row their V values
+ * must be finite (a NaN or Inf there would reach the accumulators as 0 * NaN).
  * Errors: KSA_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE before anything is launched;
  * KSA_ERR_CUDA if a launch fails.  Device-side bounded waits report through
  * ksa_last_device_status after the stream has been synchronised.

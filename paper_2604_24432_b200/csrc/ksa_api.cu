@@ -93,6 +93,21 @@ int validate_strides(const ksa_params* p)
 
 static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
+// The text kernel can read its tiles straight from the caller's interleaved tensors -- no packed
+// streams, no workspace -- when a 128-row tile is a whole number of chunks in both views and every
+// sequence is a whole number of chunks (the paper's assumption, Sec. 2.2.1), so that sequence b
+// starts at chunk aug_off_b / (k + m) of a regular [chunk, k + m] grid.  Padding rows of a partial
+// tile then hold rows of the following sequence (or zeros past the end); they are masked.
+bool direct_ok(const ksa_params* p)
+{
+    if (p->flags & KSA_FLAG_REFERENCE_KERNEL) return false;
+    const int k = p->chunk_len, m = p->summaries_per_chunk;
+    if (kTileM % k != 0 || (m > 0 && kTileN % m != 0)) return false;
+    for (int b = 0; b < p->num_seqs; ++b)
+        if ((p->cu_text_lens[b + 1] - p->cu_text_lens[b]) % k != 0) return false;
+    return true;
+}
+
 void build_layout(const ksa_params* p, HostSchedule& hs)
 {
     const int k = p->chunk_len, m = p->summaries_per_chunk;
@@ -106,6 +121,7 @@ void build_layout(const ksa_params* p, HostSchedule& hs)
         s.n_chunks = s.n_text / k;                        // only full chunks carry summaries
         s.n_summ = s.n_chunks * m;
         s.aug_off = aug;
+        s.chunk0 = (int32_t)(aug / (k + m));
         s.text_off = (int32_t)trow;
         s.summ_off = (int32_t)srow;
         s.text_pad = (int32_t)round_up(s.n_text, kTileM);
@@ -301,6 +317,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_workspace_bytes(const 
     if (!bytes) return KSA_ERR_INVALID_ARG;
     int rc = validate(p);
     if (rc != KSA_OK) return rc;
+    if (direct_ok(p)) { *bytes = 256; return KSA_OK; }     // nothing is packed
     HostSchedule hs;
     build_layout(p, hs);
     *bytes = workspace_layout(p, hs).total;
@@ -525,9 +542,25 @@ static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, 
     return KSA_OK;
 }
 
+// Chunked view of a caller tensor [rows, H, D] (element strides st, sh): dims {D, rows_per_chunk, chunks, H},
+// a box of 128 / rows_per_chunk chunks.  `base` points at the first row of the view's first chunk.
+static int encode_chunk_map(ksa_ctx* ctx, CUtensorMap* map, const void* base, int D, int rows_per_chunk, int chunk_rows,
+                            int64_t chunks, int H, int64_t st, int64_t sh)
+{
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows_per_chunk, (cuuint64_t)chunks, (cuuint64_t)H};
+    const cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)chunk_rows * st * 2, (cuuint64_t)sh * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)rows_per_chunk, (cuuint32_t)(kTileN / rows_per_chunk), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return KSA_ERR_CUDA; }
+    return KSA_OK;
+}
+
 // Kernel arguments of a whole problem (schedule already cached and uploaded in ctx).
 static KernelArgs make_args(ksa_ctx* ctx, const ksa_params* p, const void* q, const void* k, const void* v, void* out,
-                            float* lse, void* workspace, const WorkspaceLayout& wl)
+                            float* lse, void* workspace, const WorkspaceLayout& wl, bool direct = false)
 {
     const HostSchedule& hs = ctx->sched;
     char* ws = (char*)workspace;
@@ -542,6 +575,7 @@ static KernelArgs make_args(ksa_ctx* ctx, const ksa_params* p, const void* q, co
     a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
     a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
     a.r_seq = -1;
+    a.direct = direct ? 1 : 0;
     a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v;
     a.out = (uint16_t*)out; a.lse = lse;
     a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;
@@ -562,6 +596,19 @@ static int prepare_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, TextM
         ctx->tc_ready = true;
     }
     int rc;
+    if (a.direct) {
+        const int s_len = a.k + a.m;
+        const int64_t chunks = a.total_aug / s_len;
+        if ((rc = encode_chunk_map(ctx, &maps.qt, a.q, a.D, a.k, s_len, chunks, a.Hq, a.q_st, a.q_sh)) != KSA_OK) return rc;
+        if ((rc = encode_chunk_map(ctx, &maps.kt, a.kx, a.D, a.k, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
+        if ((rc = encode_chunk_map(ctx, &maps.vt, a.v, a.D, a.k, s_len, chunks, a.Hkv, a.v_st, a.v_sh)) != KSA_OK) return rc;
+        if (a.m > 0) {      // summary rows start k rows into each chunk
+            if ((rc = encode_chunk_map(ctx, &maps.ks, a.kx + (int64_t)a.k * a.k_st, a.D, a.m, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
+            return encode_chunk_map(ctx, &maps.vs, a.v + (int64_t)a.k * a.v_st, a.D, a.m, s_len, chunks, a.Hkv, a.v_st, a.v_sh);
+        }
+        maps.ks = maps.kt; maps.vs = maps.vt;    // never used: no summary tiles are scheduled
+        return KSA_OK;
+    }
     if ((rc = encode_stream_map(ctx, &maps.qt, a.qt, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
     if ((rc = encode_stream_map(ctx, &maps.kt, a.kt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
     if ((rc = encode_stream_map(ctx, &maps.vt, a.vt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
@@ -590,14 +637,17 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
     for (int i = 0; i < 5; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
     if ((rc = ensure_schedule(ctx, p, true)) != KSA_OK) return rc;
     const HostSchedule& hs = ctx->sched;
+    const bool direct = direct_ok(p);
     const WorkspaceLayout wl = workspace_layout(p, hs);
-    if (!workspace || workspace_bytes < wl.total || ((uintptr_t)workspace & 255)) return KSA_ERR_WORKSPACE;
+    if (!direct && (!workspace || workspace_bytes < wl.total || ((uintptr_t)workspace & 255))) return KSA_ERR_WORKSPACE;
 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    KernelArgs a = make_args(ctx, p, q, k, v, out, lse, workspace, wl);
+    KernelArgs a = make_args(ctx, p, q, k, v, out, lse, workspace, wl, direct);
     cudaError_t e;
-    if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 1;
+    if (!direct) {
+        if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
     if (a.m > 0 && a.max_n_summ > 0) {
         if ((e = launch_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         ctx->launches += 1;

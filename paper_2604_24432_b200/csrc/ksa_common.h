@@ -17,7 +17,7 @@ struct SeqInfo {
     int32_t summ_off;   // first row in the packed summary stream (multiple of kTileN)
     int32_t text_pad;   // padded text rows (multiple of kTileM)
     int32_t summ_pad;   // padded summary rows (multiple of kTileN)
-    int32_t reserved;
+    int32_t chunk0;     // aug_off / (k + m): first chunk of the sequence in the direct views (valid if every length is a multiple of k)
 };
 
 // One unit of work of the text-row kernel: one query tile, one or two query heads that
@@ -56,6 +56,7 @@ struct KernelArgs {
     // Row range (pack and summary kernels): r_seq < 0 means every sequence in full; otherwise only
     // sequence r_seq, packed text rows [r_text0, r_text1), summary-stream rows [r_summ0, r_summ1)
     // (pack) and summary query rows [r_summ0, r_summq1) (summary-row kernel).
+    int32_t direct;         // text kernel reads Q/K/V tiles straight from the caller's tensors (no packed streams)
     int32_t r_seq;
     int32_t r_text0, r_text1, r_summ0, r_summ1, r_summq1;
     // user tensors (bf16 as uint16)

@@ -30,6 +30,8 @@ struct WorkspaceLayout { size_t qt, kt, vt, ks, vs, total; };
 // KSA_OK or the KSA_ERR_* code describing what is wrong with p.
 int validate(const ksa_params* p);
 int validate_strides(const ksa_params* p);
+// True if the text kernel can read its tiles straight from the caller's tensors (nothing is packed).
+bool direct_ok(const ksa_params* p);
 // Fills seqs and the stream totals of hs from p (p must have passed validate).
 void build_layout(const ksa_params* p, HostSchedule& hs);
 // Fills hs.work (longest first) from p and the layout already in hs.

@@ -18,7 +18,10 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream);
 cudaError_t launch_text_ref(const KernelArgs& a, cudaStream_t stream);
 
 // Text rows, tcgen05/TMA kernel.  The five tensor maps describe the packed streams
-// as [D, rows, H] with a {64, 128, 1} box and 128-byte swizzle.
+// as [D, rows, H] with a {64, 128, 1} box and 128-byte swizzle, or (KernelArgs::direct) the
+// caller's interleaved tensors as [D, k, chunks, H] (text rows; box {64, k, 128/k, 1}) and
+// [D, m, chunks, H] starting k rows in (summary rows; box {64, m, 128/m, 1}): the box lands in
+// shared memory as the same dense 128-row tile either way.
 struct TextMaps { CUtensorMap qt, kt, vt, ks, vs; };
 cudaError_t launch_text_tc(const KernelArgs& a, const TextMaps& maps, int num_sms, cudaStream_t stream);
 // One-time per-device setup (dynamic shared memory opt-in).

@@ -193,12 +193,18 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 q_armed = true;
                 for (int t = 0; t < w.n_heads; ++t)
                     for (int h = 0; h < Cfg::kHalves; ++h)
-                        tma_load_3d(sQ + t * Cfg::kTileBytes + h * 16384, &maps.qt, bar(BAR_QFULL),
-                                    h * 64, sq.text_off + w.q_tile * kTileM, w.head0 + t);
+                        if (a.direct)
+                            tma_load_4d(sQ + t * Cfg::kTileBytes + h * 16384, &maps.qt, bar(BAR_QFULL),
+                                        h * 64, 0, sq.chunk0 + w.q_tile * (kTileM / a.k), w.head0 + t);
+                        else
+                            tma_load_3d(sQ + t * Cfg::kTileBytes + h * 16384, &maps.qt, bar(BAR_QFULL),
+                                        h * 64, sq.text_off + w.q_tile * kTileM, w.head0 + t);
                 q_phase ^= 1u;
                 for (int j = 0; j < T && alive; ++j) {
                     const bool summ = j < w.ns_tiles;
                     const int y = summ ? (sq.summ_off + j * kTileN) : (sq.text_off + (w.band_lo + j - w.ns_tiles) * kTileN);
+                    // direct views: a tile is 128/m chunks of the summary view or 128/k chunks of the text view
+                    const int zc = sq.chunk0 + (summ ? j * (kTileN / max(a.m, 1)) : (w.band_lo + j - w.ns_tiles) * (kTileN / a.k));
                     const CUtensorMap* mk = summ ? &maps.ks : &maps.kt;
                     const CUtensorMap* mv = summ ? &maps.vs : &maps.vt;
                     for (int kv = 0; kv < 2; ++kv) {
@@ -207,7 +213,10 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                         armed_mask |= 1u << stage;
                         armed_parity = (armed_parity & ~(1u << stage)) | (ring_phase << stage);
                         for (int h = 0; h < Cfg::kHalves; ++h)
-                            tma_load_3d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, y, hk);
+                            if (a.direct)
+                                tma_load_4d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, 0, zc, hk);
+                            else
+                                tma_load_3d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, y, hk);
                         if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
                     }
                 }

@@ -73,17 +73,21 @@ def test_full_size_layout_g_sampled(ctx):
     ([640], 1, 1, 100, 2, 1, 128),         # k = 1
     ([1290], 200, 3, 1, 4, 1, 128),        # chunk longer than a tile
     ([2100], 8, 1, 16, 8, 2, 128),         # several summary tiles
+    ([2048, 640, 1336], 8, 1, 16, 8, 2, 128),   # whole chunks everywhere: direct views, sequences not on tile boundaries
+    ([1024, 320], 4, 2, 9, 4, 2, 64),      # direct views with m = 2, D = 64
+    ([768], 128, 1, 2, 2, 1, 128),         # a chunk is a whole tile
 ])
 def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
     wl = synth.Workload("edge", 99, lens, Hq, Hkv, D)
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), kernel_flag)
 
 
-def test_strided_inputs_and_stream(ctx):
+@pytest.mark.parametrize("n", [900, 896])     # 896: whole chunks, tiles are read straight from the strided views
+def test_strided_inputs_and_stream(ctx, n):
     """Non-contiguous q/k/v/out views (packed QKV buffer) on a side stream."""
-    wl = synth.Workload("strided", 5, [900], 8, 2, 128)
+    wl = synth.Workload("strided", 5, [n], 8, 2, 128)
     lay = synth.Layout("s", 8, 1, 4)
-    total = orc.aug_len(900, 8, 1)
+    total = orc.aug_len(n, 8, 1)
     q, k, v = synth.make_qkv(wl, total)
     dev = torch.device("cuda", 0)
     packed = torch.zeros((total, 8 + 2 + 2 + 1, 128), dtype=torch.bfloat16, device=dev)
@@ -92,13 +96,13 @@ def test_strided_inputs_and_stream(ctx):
     outbuf = torch.zeros((total, 9, 128), dtype=torch.bfloat16, device=dev)
     out = outbuf[:, 1:]
     lse = torch.empty((8, total), dtype=torch.float32, device=dev)
-    prob = ksa.Problem([900], 8, 1, 4, 8, 2, 128, wl.scale)
+    prob = ksa.Problem([n], 8, 1, 4, 8, 2, 128, wl.scale)
     ws = torch.empty(ksa.workspace_bytes(prob), dtype=torch.uint8, device=dev)
     st = torch.cuda.Stream()
     with torch.cuda.stream(st):
         ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws, stream=st.cuda_stream)
     st.synchronize()
-    ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), [900], 8, 1, 4, wl.scale)
+    ref_out, ref_lse, _ = orc.fwd(synth.bits(q), synth.bits(k), synth.bits(v), [n], 8, 1, 4, wl.scale)
     parity.compare(out.double().cpu().numpy(), lse.double().cpu().numpy().T, ref_out, ref_lse, "strided")
     assert (outbuf[:, 0] == 0).all()
 

@@ -53,7 +53,7 @@ def test_noalloc_rejects_oversized_problem():
     ksa_build.build()
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    prob = ksa.Problem([8192], 8, 1, 128, 32, 8, 128, 0.0884)
+    prob = ksa.Problem([8189], 8, 1, 128, 32, 8, 128, 0.0884)      # not whole chunks: the packed streams are needed
     assert ksa.workspace_bytes(prob) > ksa.NOALLOC_MAX_SCRATCH_BYTES
     total = ksa.total_aug_len(prob)
     q = torch.zeros((total, 32, 128), dtype=torch.bfloat16, device=dev)
