@@ -29,7 +29,7 @@ sys.path.insert(0, ROOT)
 import numpy as np
 import torch
 
-from paper_2604_24432_b200 import synth
+from paper_2604_24432_b200 import dist_utils, synth
 
 METRIC = "KSA attn fwd visible TFLOP/s & text tok/s at 128K, % of B200 BF16 peak"
 
@@ -189,8 +189,7 @@ def run_ours(args):
         ksa_build.build()
     wl, layout = workload_and_layout(args)
     if world > 1:   # independent batch per rank
-        import dataclasses
-        wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+        wl = dist_utils.rank_workload(wl, rank)
     prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
     total = ksa.total_aug_len(prob)
     pairs = ksa.visible_pairs(prob)
@@ -233,14 +232,10 @@ def run_ours(args):
     total_ms = ev[0].elapsed_time(ev[args.steps])
     ctx.enable_kernel_timing(False)
     assert ctx.device_status() == 0, "device-side wait gave up"
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = dist_utils.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
-    tok_s = world * n_text / (ms_per_step * 1e-3)
+    value = dist_utils.aggregate_rate(flops, world, ms_per_step) / 1e12
+    tok_s = dist_utils.aggregate_rate(n_text, world, ms_per_step)
 
     # ---- end to end through the host entry point ----------------------------------------
     e2e = None
@@ -258,11 +253,7 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = dist_utils.max_over_ranks(e2e_ms, dev)
         h2d = qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2
         d2h = out_h.numel() * 2 + lse_h.numel() * 4
         e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
