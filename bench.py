@@ -345,17 +345,36 @@ def run_decode(args):
         pos = step(pos)
     torch.cuda.synchronize()
     assert ctx.device_status() == 0
+    steps = max(k, (steps // k) * k)            # whole chunks: k text steps and the chunk's summary step
     launches0 = ctx.launch_count()
     bytes_read = 0
+    for i in range(steps):
+        lo, hi = ksa.cache_slice(spec, pos + i, False)
+        bytes_read += B * Hkv * (hi - lo) * D * 2 * 2
+        if (pos + i + 1) % k == 0:
+            bytes_read += B * Hkv * (k + 1) * D * 2 * 2
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph = None
+    if not args.no_graph:
+        # the step kernels take everything that changes from the device-side state, so one chunk's worth
+        # of steps is captured once and replayed (no launch gaps between the four kernels of a step)
+        launches_per_chunk = ctx.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            p_ = pos
+            for _ in range(k):
+                p_ = step(p_)
+        launches_per_chunk = ctx.launch_count() - launches_per_chunk
+        stream = torch.cuda.current_stream(dev)
     with ClockSampler(local) as clocks:
         e0.record(stream)
-        for _ in range(steps):
-            lo, hi = ksa.cache_slice(spec, pos, False)
-            bytes_read += B * Hkv * (hi - lo) * D * 2 * 2
-            if (pos + 1) % k == 0:
-                bytes_read += B * Hkv * (k + 1) * D * 2 * 2
-            pos = step(pos)
+        if graph is not None:
+            for _ in range(steps // k):
+                graph.replay()
+            pos += steps
+        else:
+            for _ in range(steps):
+                pos = step(pos)
         e1.record(stream)
         torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
@@ -371,8 +390,10 @@ def run_decode(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)",
         "config": {"workload": f"decode, {B} sequences at {ctx_len} cached text tokens each", "layout": f"P: k={k} m=1 C={C}",
                    "heads": f"{Hq}q/{Hkv}kv", "head_dim": D, "cache_gb": cache_gb,
-                   "l2_policy": "the cache slices read per step are larger than L2 (no flush)", "parallelism": "1 GPU"},
-        "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
+                   "l2_policy": "the cache slices read per step are larger than L2 (no flush)", "parallelism": "1 GPU",
+                   "launch": "CUDA graph of one chunk (k text steps + its summary step), replayed" if graph is not None else "plain launches"},
+        "clocks": clocks.summary(),
+        "gpu_launches": int(launches_per_chunk * (steps // k)) if graph is not None else int(ctx.launch_count() - launches0),
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                      "traffic": None, "peak_source": f"of {peaks['source']} (copy bandwidth)",
                      "kernel": "ksa_decode_attn_kernel (+ append, merge, commit)",
@@ -406,6 +427,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
     ap.add_argument("--decode-batch", type=int, default=32)
+    ap.add_argument("--no-graph", action="store_true", help="decode: plain launches instead of a replayed CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -405,11 +405,22 @@ static int validate_cache(const ksa_cache_params* p)
     return KSA_OK;
 }
 
+// Splits of a slice: the grid (splits x batch x KV heads) should fill whole waves of the 2 x 148
+// resident CTAs (two per SM) -- the smallest split count of at least two waves that wastes less
+// than 5 % of the last wave, or the most efficient one up to 32.
 static int decode_splits(const ksa_cache_params* p)
 {
-    const int64_t units = (int64_t)p->batch * p->num_kv_heads;
-    int64_t n = (2 * 148 + units - 1) / units;          // about two CTAs per SM in flight
-    return (int)std::max<int64_t>(1, std::min<int64_t>(64, n));
+    const int64_t units = (int64_t)p->batch * p->num_kv_heads, slots = 2 * 148;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int n = 1; n <= 32; ++n) {
+        const int64_t total = units * n;
+        if (total < 2 * slots && n < 32) continue;
+        const double eff = (double)total / (double)(((total + slots - 1) / slots) * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = n; }
+        if (eff >= 0.95) break;
+    }
+    return best;
 }
 
 KSA_API int64_t ksa_cache_rows(const ksa_cache_params* p)
