@@ -1,5 +1,5 @@
 /*
- * ksa_oracle.c -- plain CPU oracle for Kwai Summary Attention (KSA) forward.
+ * ksa_oracle.c -- plain CPU oracle for Kwai Summary Attention (KSA): forward and gradients.
  *
  * TEST INFRASTRUCTURE ONLY (see ksa_oracle.h).  Plain C, fp64 arithmetic on the
  * exact bf16 input values, explicit mask row per query, no tiling, no skipping of
@@ -221,4 +221,97 @@ int ksa_oracle_fwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v,
     }
     free(aug_off);
     return bad ? -1 : 0;
+}
+
+/* Softmax weights of row pq of a sequence (head h) over its explicit mask row: x[] receives
+ * p_j on visible positions (untouched elsewhere), the return value is the row's output o (in acc). */
+static void row_weights(const uint16_t* q, const uint16_t* kk, const uint16_t* v, int64_t base, int64_t L,
+                        int64_t g, int32_t h, int32_t hk, int32_t Hq, int32_t Hkv, int32_t D, double scale,
+                        const uint8_t* mask, double* x, double* acc)
+{
+    const uint16_t* qrow = q + ((size_t)g * Hq + h) * (size_t)D;
+    double M = -INFINITY;
+    for (int64_t pk = 0; pk < L; ++pk) {
+        if (!mask[pk]) continue;
+        const uint16_t* krow = kk + ((size_t)(base + pk) * Hkv + hk) * (size_t)D;
+        double dot = 0.0;
+        for (int32_t d = 0; d < D; ++d) dot += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+        x[pk] = scale * dot;
+        if (x[pk] > M) M = x[pk];
+    }
+    double l = 0.0;
+    for (int64_t pk = 0; pk < L; ++pk)
+        if (mask[pk]) { x[pk] = exp(x[pk] - M); l += x[pk]; }
+    for (int32_t d = 0; d < D; ++d) acc[d] = 0.0;
+    for (int64_t pk = 0; pk < L; ++pk) {
+        if (!mask[pk]) continue;
+        x[pk] /= l;                                   /* p_j */
+        const uint16_t* vrow = v + ((size_t)(base + pk) * Hkv + hk) * (size_t)D;
+        for (int32_t d = 0; d < D; ++d) acc[d] += x[pk] * bf16_to_double(vrow[d]);
+    }
+}
+
+int ksa_oracle_bwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v, const uint16_t* dout,
+                   int32_t num_seqs, const int32_t* cu_text_lens,
+                   int32_t k, int32_t m, int32_t C,
+                   int32_t Hq, int32_t Hkv, int32_t D, double scale, uint32_t flags,
+                   double* dq, double* dk, double* dv)
+{
+    if (!q || !kk || !v || !dout || !cu_text_lens || !dq || !dk || !dv) return -1;
+    if (num_seqs < 1 || k < 1 || m < 0 || C < 0 || Hq < 1 || Hkv < 1 || D < 1 || Hq % Hkv != 0) return -1;
+    const int32_t G = Hq / Hkv;
+    int64_t total_aug = 0, max_L = 1;
+    for (int32_t b = 0; b < num_seqs; ++b) {
+        int64_t L = ksa_oracle_aug_len((int64_t)cu_text_lens[b + 1] - cu_text_lens[b], k, m);
+        if (L < 0) return -1;
+        total_aug += L;
+        if (L > max_L) max_L = L;
+    }
+    memset(dq, 0, sizeof(double) * (size_t)total_aug * Hq * D);
+    memset(dk, 0, sizeof(double) * (size_t)total_aug * Hkv * D);
+    memset(dv, 0, sizeof(double) * (size_t)total_aug * Hkv * D);
+
+    /* One KV head per task: rows are walked in order, so the sums into dk / dv of that head need no
+     * locking and always add in the same order. */
+#pragma omp parallel
+    {
+        uint8_t* mask = (uint8_t*)malloc((size_t)max_L);
+        double* p = (double*)malloc(sizeof(double) * (size_t)max_L);
+        double* o = (double*)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (int32_t hk = 0; hk < Hkv; ++hk) {
+            int64_t base = 0;
+            for (int32_t b = 0; b < num_seqs; ++b) {
+                const int64_t n = (int64_t)cu_text_lens[b + 1] - cu_text_lens[b];
+                const int64_t L = ksa_oracle_aug_len(n, k, m);
+                for (int64_t pq = 0; pq < L; ++pq) {
+                    ksa_oracle_mask_row(n, k, m, C, flags, pq, mask);
+                    const int64_t g = base + pq;
+                    for (int32_t h = hk * G; h < (hk + 1) * G; ++h) {
+                        row_weights(q, kk, v, base, L, g, h, hk, Hq, Hkv, D, scale, mask, p, o);
+                        const uint16_t* qrow = q + ((size_t)g * Hq + h) * (size_t)D;
+                        const uint16_t* drow = dout + ((size_t)g * Hq + h) * (size_t)D;
+                        double delta = 0.0;                               /* <dO_i, o_i> */
+                        for (int32_t d = 0; d < D; ++d) delta += bf16_to_double(drow[d]) * o[d];
+                        double* dqrow = dq + ((size_t)g * Hq + h) * (size_t)D;
+                        for (int64_t pk = 0; pk < L; ++pk) {
+                            if (!mask[pk]) continue;
+                            const size_t kvoff = ((size_t)(base + pk) * Hkv + hk) * (size_t)D;
+                            double dP = 0.0;                              /* <dO_i, v_j> */
+                            for (int32_t d = 0; d < D; ++d) dP += bf16_to_double(drow[d]) * bf16_to_double(v[kvoff + d]);
+                            const double dS = p[pk] * (dP - delta);
+                            for (int32_t d = 0; d < D; ++d) {
+                                dv[kvoff + d] += p[pk] * bf16_to_double(drow[d]);
+                                dk[kvoff + d] += scale * dS * bf16_to_double(qrow[d]);
+                                dqrow[d] += scale * dS * bf16_to_double(kk[kvoff + d]);
+                            }
+                        }
+                    }
+                }
+                base += L;
+            }
+        }
+        free(mask); free(p); free(o);
+    }
+    return 0;
 }

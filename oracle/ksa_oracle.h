@@ -87,6 +87,25 @@ int ksa_oracle_fwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v,
                    const int64_t* rows, int64_t n_rows,
                    double* out, double* lse, int64_t* count);
 
+/*
+ * Gradients of the same operator (what a training step needs; Sec. 2.3 calls the block-sparse
+ * kernel the one "for training and prefill"), in fp64 from bf16 inputs.  With p_ij the softmax
+ * weights of row i over its visible keys, o_i = sum_j p_ij v_j and dO given:
+ *   dV_j = sum_i p_ij dO_i            dP_ij = <dO_i, v_j>          delta_i = <dO_i, o_i>
+ *   dS_ij = p_ij (dP_ij - delta_i)    dQ_i = scale sum_j dS_ij k_j  dK_j = scale sum_i dS_ij q_i
+ * (the textbook gradient of softmax(scale Q K^T + M) V; sums over i run over the rows that see j,
+ * and for grouped heads dK, dV add up the G query heads of a KV head).
+ *   q, kk, v, cu_text_lens, k, m, C, Hq, Hkv, D, scale, flags   as in ksa_oracle_fwd
+ *   dout   [total_aug, Hq, D] bf16 bit patterns
+ *   dq     [total_aug, Hq, D] fp64;  dk, dv [total_aug, Hkv, D] fp64 (every entry written)
+ * Returns 0, or -1 on bad arguments.
+ */
+int ksa_oracle_bwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v, const uint16_t* dout,
+                   int32_t num_seqs, const int32_t* cu_text_lens,
+                   int32_t k, int32_t m, int32_t C,
+                   int32_t Hq, int32_t Hkv, int32_t D, double scale, uint32_t flags,
+                   double* dq, double* dk, double* dv);
+
 /* Threads the OpenMP loops will use. */
 int ksa_oracle_num_threads(void);
 

@@ -63,6 +63,7 @@ def _load():
     lib.ksa_oracle_fwd.restype = ctypes.c_int
     lib.ksa_oracle_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, i32,
                                    ctypes.c_double, u32, vp, i64, vp, vp, vp]
+    lib.ksa_oracle_bwd.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, i32, ctypes.c_double, u32, vp, vp, vp]
     lib.ksa_oracle_num_threads.restype = ctypes.c_int
     _lib = lib
     return lib
@@ -150,3 +151,24 @@ def fwd(q_bits, k_bits, v_bits, text_lens, k, m, C, scale, flags=0, rows=None):
     if rc != 0:
         raise ValueError("ksa_oracle_fwd: bad argument")
     return out, lse, cnt
+
+
+def bwd(q_bits, k_bits, v_bits, dout_bits, text_lens, k, m, C, scale, flags=0):
+    """Gradients (dq, dk, dv) in fp64 for the upstream gradient dout (bf16 bit patterns), all rows."""
+    lib = _load()
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    k_bits = np.ascontiguousarray(k_bits, dtype=np.uint16)
+    v_bits = np.ascontiguousarray(v_bits, dtype=np.uint16)
+    dout_bits = np.ascontiguousarray(dout_bits, dtype=np.uint16)
+    total, Hq, D = q_bits.shape
+    Hkv = k_bits.shape[1]
+    cu = np.concatenate([[0], np.cumsum(np.asarray(text_lens, dtype=np.int64))]).astype(np.int32)
+    dq = np.empty((total, Hq, D), dtype=np.float64)
+    dk = np.empty((total, Hkv, D), dtype=np.float64)
+    dv = np.empty((total, Hkv, D), dtype=np.float64)
+    rc = lib.ksa_oracle_bwd(q_bits.ctypes.data, k_bits.ctypes.data, v_bits.ctypes.data, dout_bits.ctypes.data,
+                            len(text_lens), cu.ctypes.data, k, m, C, Hq, Hkv, D, float(scale), flags,
+                            dq.ctypes.data, dk.ctypes.data, dv.ctypes.data)
+    if rc != 0:
+        raise ValueError("ksa_oracle_bwd: bad arguments")
+    return dq, dk, dv
