@@ -147,6 +147,27 @@ int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v,
                  void* out, float* lse, void* workspace, size_t workspace_bytes,
                  const ksa_params* p, void* cuda_stream);
 
+/* ---- backward ----------------------------------------------------------------------- */
+/* Bytes of DEVICE workspace ksa_attn_bwd needs for this problem. */
+int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
+/*
+ * Gradients of ksa_attn_fwd (the kernel of Sec. 2.3 is the one "for training and prefill"):
+ * with P the softmax weights of the forward pass (recomputed from q, k and lse),
+ *   dV = P^T dO,  dP = dO V^T,  dS = P o (dP - rowsum(dO o O)),  dQ = scale dS K,  dK = scale dS^T Q
+ * under the same mask (Eq. 3 for text rows, own chunk for summary rows); for grouped heads dK and
+ * dV add up the query heads of their KV head.
+ *   q, k, v, out, lse   DEVICE, the tensors given to / written by ksa_attn_fwd (same p)
+ *   dout                DEVICE bf16, gradient w.r.t. out, layout and strides of out
+ *   dq                  DEVICE bf16, layout and strides of q; every row is written
+ *   dk, dv              DEVICE bf16, layouts and strides of k and v; every row is written
+ *   workspace           DEVICE, >= ksa_bwd_workspace_bytes, 256-byte aligned, scratch
+ * Asynchronous on cuda_stream.  KSA_FLAG_REFERENCE_KERNEL is not accepted here.
+ * Errors as for ksa_attn_fwd.
+ */
+int ksa_attn_bwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                 const void* dout, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                 const ksa_params* p, void* cuda_stream);
+
 /* Bytes of DEVICE staging ksa_attn_fwd_host needs (q, k, v, out, lse images plus the
  * workspace of ksa_attn_fwd). */
 int ksa_host_staging_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);

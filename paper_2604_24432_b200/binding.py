@@ -27,7 +27,7 @@ KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
 EXPORTS = [
     "ksa_create", "ksa_destroy", "ksa_aug_len", "ksa_total_aug_len", "ksa_workspace_bytes",
     "ksa_visible_pairs", "ksa_attn_fwd", "ksa_host_staging_bytes", "ksa_attn_fwd_host",
-    "ksa_attn_fwd_noalloc",
+    "ksa_attn_fwd_noalloc", "ksa_bwd_workspace_bytes", "ksa_attn_bwd",
     "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
     "ksa_last_cuda_error", "ksa_launch_count", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
     "ksa_strerror",
@@ -99,6 +99,8 @@ def lib():
     L.ksa_host_staging_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, pp, vp]
+    L.ksa_bwd_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
+    L.ksa_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
     L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.ksa_clear_device_status.argtypes = [vp]
@@ -190,6 +192,13 @@ def workspace_bytes(prob: Problem) -> int:
     return int(n.value)
 
 
+def bwd_workspace_bytes(prob: Problem) -> int:
+    p = prob.params()
+    n = ctypes.c_size_t()
+    _check(lib().ksa_bwd_workspace_bytes(None, ctypes.byref(p), ctypes.byref(n)), "ksa_bwd_workspace_bytes")
+    return int(n.value)
+
+
 def host_staging_bytes(prob: Problem) -> int:
     p = prob.params()
     n = ctypes.c_size_t()
@@ -245,6 +254,17 @@ class Context:
         _check(lib().ksa_attn_fwd(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                   lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                   ctypes.byref(p), stream), "ksa_attn_fwd")
+
+    def attn_bwd(self, prob: Problem, q, k, v, out, lse, dout, dq, dk, dv, workspace, stream: Optional[int] = None):
+        """ksa_attn_bwd on torch CUDA tensors (dout like out, dq like q, dk / dv like k / v)."""
+        import torch
+        p = prob.params(q, k, v, out)
+        assert dout.stride() == out.stride() and dq.stride() == q.stride() and dk.stride() == k.stride() and dv.stride() == v.stride()
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        _check(lib().ksa_attn_bwd(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                  dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), ctypes.byref(p), stream), "ksa_attn_bwd")
 
     def attn_fwd_host(self, prob: Problem, q, k, v, out, lse, staging, stream: Optional[int] = None):
         """ksa_attn_fwd_host: q, k, v, out, lse are contiguous HOST tensors (pinned recommended)."""

@@ -8,6 +8,7 @@
 
 #include "../../include/ksa.h"
 #include "ksa_host.h"
+#include "ksa_bwd.h"
 #include "ksa_launch.h"
 
 using namespace ksa;
@@ -662,6 +663,94 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
 
 // Number of row chunks the host entry point aims for (upload / compute / download stages).
 static constexpr int kHostPipelineChunks = 8;
+
+// ---------------------------------------------------------------------------------------
+// backward
+// ---------------------------------------------------------------------------------------
+struct BwdLayout { WorkspaceLayout fwd; size_t dot, lse_t, delta_t, dkt, dvt, dks, dvs, total; };
+static BwdLayout bwd_layout(const ksa_params* p, const HostSchedule& hs)
+{
+    BwdLayout b{};
+    b.fwd = workspace_layout(p, hs);
+    size_t off = b.fwd.total;
+    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
+    const size_t D = (size_t)p->head_dim;
+    b.dot = take((size_t)p->num_q_heads * hs.text_rows * D * 2);
+    b.lse_t = take((size_t)p->num_q_heads * hs.text_rows * 4);
+    b.delta_t = take((size_t)p->num_q_heads * hs.text_rows * 4);
+    b.dkt = take((size_t)p->num_kv_heads * hs.text_rows * D * 4);
+    b.dvt = take((size_t)p->num_kv_heads * hs.text_rows * D * 4);
+    b.dks = take((size_t)p->num_kv_heads * hs.summ_rows * D * 4);
+    b.dvs = take((size_t)p->num_kv_heads * hs.summ_rows * D * 4);
+    b.total = off;
+    return b;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_bwd_workspace_bytes(const ksa_ctx*, const ksa_params* p, size_t* bytes)
+{
+    if (!bytes) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    HostSchedule hs;
+    build_layout(p, hs);
+    *bytes = bwd_layout(p, hs).total;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, const void* out,
+                            const float* lse, const void* dout, void* dq, void* dk, void* dv, void* workspace,
+                            size_t workspace_bytes, const ksa_params* p, void* cuda_stream)
+{
+    if (!ctx || !q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = validate_strides(p)) != KSA_OK) return rc;
+    if (p->flags & KSA_FLAG_REFERENCE_KERNEL) return KSA_ERR_INVALID_ARG;
+    const uintptr_t ptrs[9] = {(uintptr_t)q, (uintptr_t)k, (uintptr_t)v, (uintptr_t)out, (uintptr_t)lse, (uintptr_t)dout,
+                               (uintptr_t)dq, (uintptr_t)dk, (uintptr_t)dv};
+    for (int i = 0; i < 9; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
+    if ((rc = ensure_schedule(ctx, p, true)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    const BwdLayout bl = bwd_layout(p, hs);
+    if (!workspace || workspace_bytes < bl.total || ((uintptr_t)workspace & 255)) return KSA_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* ws = (char*)workspace;
+    cudaError_t e;
+    static bool bwd_ready = false;
+    if (!bwd_ready) {
+        if ((e = setup_bwd()) != cudaSuccess) return cuda_fail(ctx, e);
+        bwd_ready = true;
+    }
+    // packed streams of the forward pass (text Q, K, V and summary K, V)
+    KernelArgs fa = make_args(ctx, p, q, k, v, dq /* unused */, const_cast<float*>(lse), workspace, bl.fwd);
+    if ((e = launch_pack(fa, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    BwdArgs a{};
+    a.seqs = ctx->d_seqs; a.num_seqs = p->num_seqs;
+    a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.C = p->window_chunks;
+    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.flags = p->flags; a.scale = p->softmax_scale; a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+    a.total_aug = hs.total_aug; a.text_rows = hs.text_rows; a.summ_rows = hs.summ_rows;
+    a.max_text_pad = hs.max_text_pad; a.max_summ_pad = hs.max_summ_pad; a.max_n_summ = hs.max_n_summ;
+    a.q = (const uint16_t*)q; a.kx = (const uint16_t*)k; a.v = (const uint16_t*)v; a.out = (const uint16_t*)out;
+    a.dout = (const uint16_t*)dout; a.lse = lse;
+    a.dq = (uint16_t*)dq; a.dk = (uint16_t*)dk; a.dv = (uint16_t*)dv;
+    a.q_st = a.dq_st = p->q_stride_tok; a.q_sh = a.dq_sh = p->q_stride_head;
+    a.k_st = a.dk_st = p->k_stride_tok; a.k_sh = a.dk_sh = p->k_stride_head;
+    a.v_st = a.dv_st = p->v_stride_tok; a.v_sh = a.dv_sh = p->v_stride_head;
+    a.o_st = a.do_st = p->o_stride_tok; a.o_sh = a.do_sh = p->o_stride_head;
+    a.qt = fa.qt; a.kt = fa.kt; a.vt = fa.vt; a.ks = fa.ks; a.vs = fa.vs;
+    a.dot = (uint16_t*)(ws + bl.dot); a.lse_t = (float*)(ws + bl.lse_t); a.delta_t = (float*)(ws + bl.delta_t);
+    a.dkt = (float*)(ws + bl.dkt); a.dvt = (float*)(ws + bl.dvt); a.dks = (float*)(ws + bl.dks); a.dvs = (float*)(ws + bl.dvs);
+    // the four accumulators are contiguous in the workspace: one clear
+    if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_bwd_dq(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 5 + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
+    return KSA_OK;
+}
 
 struct StagingLayout { size_t q, k, v, out, lse, ws, ws_bytes, total; };
 static int staging_layout(const ksa_params* p, StagingLayout& s)

@@ -1,0 +1,41 @@
+// Internal interface of the backward pass (kernel arguments and launchers).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "ksa_common.h"
+
+namespace ksa {
+
+struct BwdArgs {
+    const SeqInfo* seqs;
+    int32_t num_seqs;
+    int32_t k, m, C, Hq, Hkv, D;
+    uint32_t flags;
+    float scale, scale_log2;
+    int64_t total_aug, text_rows, summ_rows;
+    int32_t max_text_pad, max_summ_pad, max_n_summ;
+    // caller tensors (bf16 bit patterns; lse fp32 [Hq, total_aug])
+    const uint16_t* q; const uint16_t* kx; const uint16_t* v; const uint16_t* out; const uint16_t* dout; const float* lse;
+    uint16_t* dq; uint16_t* dk; uint16_t* dv;
+    int64_t q_st, q_sh, k_st, k_sh, v_st, v_sh, o_st, o_sh, do_st, do_sh, dq_st, dq_sh, dk_st, dk_sh, dv_st, dv_sh;
+    // workspace: packed streams of the forward pass, packed dO, per-row scalars, fp32 accumulators
+    const uint16_t* qt; const uint16_t* kt; const uint16_t* vt; const uint16_t* ks; const uint16_t* vs;
+    uint16_t* dot;              // [Hq][text_rows][D]
+    float* lse_t;               // [Hq][text_rows], times log2(e); +inf on padding rows
+    float* delta_t;             // [Hq][text_rows], <dO, O>
+    float* dkt; float* dvt;     // [Hkv][text_rows][D] fp32
+    float* dks; float* dvs;     // [Hkv][summ_rows][D] fp32
+};
+
+// Packs the text rows of dO, lse (in log2 units) and delta = <dO, O>.
+cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream);
+// Summary query rows: their dQ rows directly, their dK / dV contributions into the accumulators.
+cudaError_t launch_bwd_summary(const BwdArgs& a, cudaStream_t stream);
+// Text query rows: dQ (written directly), then dK / dV into the accumulators.
+cudaError_t launch_bwd_dq(const BwdArgs& a, cudaStream_t stream);
+cudaError_t launch_bwd_dkv(const BwdArgs& a, cudaStream_t stream);
+// Accumulators -> bf16 dk / dv at the augmented positions.
+cudaError_t launch_bwd_finish(const BwdArgs& a, cudaStream_t stream);
+cudaError_t setup_bwd();
+
+}  // namespace ksa

@@ -1,0 +1,67 @@
+"""GPU parity of the backward pass (dQ, dK, dV) against the oracle's fp64 gradients.
+
+Tolerances: the gradients are bf16 and the kernel feeds bf16 probabilities / dS to the tensor
+cores, so every product carries a relative error of about 2^-9; with magnitudes that vary by
+orders between rows the bound is relative to the tensor's scale:
+max |err| <= 2e-2 * max |ref| + 1e-5 and mean |err| <= 1e-2 * mean |ref| + 1e-5."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ksa_oracle as orc
+from paper_2604_24432_b200 import binding as ksa
+from paper_2604_24432_b200 import build as ksa_build
+from paper_2604_24432_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    ksa_build.build()
+    c = ksa.Context(0)
+    yield c
+    c.close()
+
+
+def _check(name, got, ref):
+    assert np.isfinite(got).all(), name
+    err = np.abs(got - ref)
+    # 1e-5: floor for gradients that are exactly zero (a row with a single visible key has dS = 0)
+    assert err.max() <= 2e-2 * np.abs(ref).max() + 1e-5, (name, err.max(), np.abs(ref).max())
+    assert err.mean() <= 1e-2 * np.abs(ref).mean() + 1e-5, (name, err.mean(), np.abs(ref).mean())
+
+
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D,flags", [
+    ([300, 77], 8, 1, 2, 4, 2, 128, 0),
+    ([1000], 8, 1, 16, 8, 2, 128, 0),                 # several summary tiles, G = 4
+    ([520, 130], 3, 2, 5, 6, 2, 64, 0),               # k does not divide the tile, m = 2, G = 3, D = 64
+    ([700], 16, 0, 7, 4, 4, 128, 0),                  # no summaries
+    ([450], 8, 1, 3, 4, 1, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
+    ([1], 8, 1, 2, 2, 2, 64, 0),
+    ([2100, 640], 8, 1, 16, 8, 2, 128, 0),            # several query segments per summary key tile
+])
+def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
+    wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
+    total = sum(orc.aug_len(n, k, m) for n in lens)
+    q, kk, v = synth.make_qkv(wl, total)
+    g = torch.Generator("cpu").manual_seed(77)
+    dout = torch.randn((total, Hq, D), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    dev = torch.device("cuda", 0)
+    prob = ksa.Problem(lens, k, m, C, Hq, Hkv, D, wl.scale, flags)
+    qd, kd, vd, gd = q.to(dev), kk.to(dev), v.to(dev), dout.to(dev)
+    out = torch.empty_like(qd); lse = torch.empty((Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx.clear_device_status()
+    ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws)
+    dq = torch.full_like(qd, 7.0); dk = torch.full_like(kd, 7.0); dv = torch.full_like(vd, 7.0)
+    wsb = torch.full((ksa.bwd_workspace_bytes(prob),), 0xFF, dtype=torch.uint8, device=dev)    # NaN patterns
+    for _ in range(2):                          # twice: the accumulators must be cleared by the call itself
+        ctx.attn_bwd(prob, qd, kd, vd, out, lse, gd, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    oflags = orc.SUMMARY_TEXT_ONLY if flags else 0
+    rdq, rdk, rdv = orc.bwd(synth.bits(q), synth.bits(kk), synth.bits(v), synth.bits(dout), lens, k, m, C, wl.scale, oflags)
+    _check("dq", dq.double().cpu().numpy(), rdq)
+    _check("dk", dk.double().cpu().numpy(), rdk)
+    _check("dv", dv.double().cpu().numpy(), rdv)
