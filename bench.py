@@ -404,6 +404,66 @@ def run_decode(args):
     return 0
 
 
+# ---------------------------------------------------------------------------------------
+# backward pass (secondary line)
+# ---------------------------------------------------------------------------------------
+def run_backward(args):
+    """python bench.py --backward [--workload 32k]: forward once, then the backward pass timed.  Visible FLOPs of
+    the backward pass = 2.5 x the forward's (five products of the same visible pairs instead of two)."""
+    from paper_2604_24432_b200 import binding as ksa
+    from paper_2604_24432_b200 import build as ksa_build
+    rank, world, local = dist_env()
+    if rank != 0:
+        return 0
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ksa_build.build()
+    wl, layout = workload_and_layout(args)
+    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total = ksa.total_aug_len(prob)
+    flops = 2.5 * 4.0 * wl.D * wl.Hq * ksa.visible_pairs(prob)
+    qh, kh, vh = synth.make_qkv(wl, total)
+    q, k, v = qh.to(dev), kh.to(dev), vh.to(dev)
+    del qh, kh, vh
+    g = torch.Generator(device=dev).manual_seed(9)
+    dout = torch.randn((total, wl.Hq, wl.D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty_like(q); lse = torch.empty((wl.Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx = ksa.Context(local)
+    ctx.attn_fwd(prob, q, k, v, out, lse, ws)
+    del ws
+    dq = torch.empty_like(q); dk = torch.empty_like(k); dv = torch.empty_like(v)
+    wsb = torch.empty(ksa.bwd_workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    for _ in range(max(args.warmup, 3)):
+        ctx.attn_bwd(prob, q, k, v, out, lse, dout, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record(stream)
+        for _ in range(args.steps):
+            ctx.attn_bwd(prob, q, k, v, out, lse, dout, dq, dk, dv, wsb)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    assert ctx.device_status() == 0
+    peaks = load_peaks()
+    val = flops / (ms * 1e-3) / 1e12
+    line = {
+        "metric": "KSA attn bwd visible TFLOP/s (2.5 x forward FLOPs)", "value": val, "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)", "config": base_config(wl, layout, 1),
+        "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
+        "roofline": {"bound": "tensor", "achieved": val, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                     "frac": val / peaks["bf16_sustained"], "traffic": None,
+                     "peak_source": f"of {peaks['source']} (sustained bf16 GEMM)", "kernel": "ksa_bwd_dq_kernel + ksa_bwd_dkv_kernel (mma.sync; whole step)"},
+        "e2e": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def summary_pairs(wl, layout):
     """Visible pairs of the summary rows (they run in their own small kernel)."""
     tot = 0
@@ -427,12 +487,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
     ap.add_argument("--decode-batch", type=int, default=32)
+    ap.add_argument("--backward", action="store_true", help="secondary line: the backward pass")
     ap.add_argument("--no-graph", action="store_true", help="decode: plain launches instead of a replayed CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     if args.decode:
         return run_decode(args)
+    if args.backward:
+        return run_backward(args)
     return run_ours(args)
 
 
