@@ -42,6 +42,7 @@ constexpr int kTraceEvents = 8192;
 constexpr int kTraceRoles = 12;             // 0 MMA issuer, 1-2 softmax row 0 of tile 0/1, 3 producer, 4-11 per-warp arrivals
 __device__ uint2 g_trace[2][kTraceRoles][kTraceEvents];
 __device__ uint32_t g_trace_cnt[2][kTraceRoles];
+__device__ unsigned long long g_cta_span[2][256];   // start / end of every CTA (globaltimer, ns)
 #define KSA_TR(role, id)                                                                           \
     do {                                                                                           \
         if (tr_slot >= 0 && tr_n < (uint32_t)kTraceEvents) {                                       \
@@ -135,6 +136,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
 #ifdef KSA_TRACE
     const int tr_slot = (blockIdx.x == 0) ? 0 : ((blockIdx.x == 100) ? 1 : -1);
     uint32_t tr_n = 0;
+    if (tid == 0 && blockIdx.x < 256) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); g_cta_span[0][blockIdx.x] = t_; }
 #endif
 
     if (tid == 0) {
@@ -264,9 +266,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 if (!bounded_wait(kv_full(stage), ring_phase, abort_addr, a.status, kStatusWaitKvFull)) break;
                 tc_fence_after();
                 for (int t = 0; t < nh; ++t) { issue_qk(t, stage); tc_commit(bar(BAR_SFULL + t)); }
-                tc_commit(kv_empty(stage));
                 if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
-                if (T == 1) tc_commit(bar(BAR_QEMPTY));
                 for (int j = 0; j < T && alive; ++j) {
                     const int vstage = stage; const uint32_t vphase = ring_phase;
                     if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
@@ -298,11 +298,6 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                         }
                     }
                     if (!alive) break;
-                    tc_commit(kv_empty(vstage));
-                    if (j + 1 < T) {
-                        tc_commit(kv_empty(kstage));
-                        if (j + 1 == T - 1) tc_commit(bar(BAR_QEMPTY));
-                    }
                 }
             }
             // drain the tensor pipe before TMEM is released
@@ -322,11 +317,22 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
         uint32_t sf_phase = 0, of_phase = 0;
         const int s_len = a.k + a.m;
         bool alive = true;
+        // Shared-memory stages (and the Q tiles) are handed back to the producer by one thread of the
+        // LAST query tile's warpgroup: tcgen05 operations of the issuing thread complete in order, so
+        // its s_full for key tile j says that every product issued before it has finished reading --
+        // K(j) and V(j-1) for both query tiles.  This keeps those signals out of the MMA thread's
+        // instruction stream.  Every thread follows the ring position (two stages per key tile).
+        int rel_stage = 0;
+        auto release_next = [&]() {
+            mbar_arrive(kv_empty(rel_stage));
+            if (++rel_stage == Cfg::kStages) rel_stage = 0;
+        };
         for (int r = 0; alive; ++r) {
             const int idx = item_index(r);
             if (idx >= a.num_work) break;
             const WorkItem w = a.work[idx];
-            if (t >= w.n_heads) continue;
+            if (t >= w.n_heads) { rel_stage = (rel_stage + 2 * (w.ns_tiles + (w.band_hi - w.band_lo + 1))) % Cfg::kStages; continue; }
+            const bool releaser = (t == w.n_heads - 1) && (tid & 127) == 0;
             const SeqInfo sq = a.seqs[w.seq];
             const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
             const int i_raw = w.q_tile * kTileM + row;
@@ -343,6 +349,13 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { alive = false; break; }
                 sf_phase ^= 1u;
+                if (releaser) {
+                    if (j > 0) release_next();                   // V(j-1)
+                    release_next();                              // K(j)
+                    if (j == T - 1) mbar_arrive(bar(BAR_QEMPTY));
+                } else if ((tid & 127) == 0) {
+                    rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
+                }
                 if (row == 0) KSA_TR(1 + t, 1);
                 tc_fence_after();
                 uint32_t s[128];
@@ -444,6 +457,8 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             of_phase ^= 1u;
+            if (releaser) release_next();                        // V(T-1)
+            else if ((tid & 127) == 0) rel_stage = (rel_stage + 1) % Cfg::kStages;
             tc_fence_after();
             const float inv_l = 1.f / l_run;
             const int h = w.head0 + t;
@@ -473,10 +488,19 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
 
     tc_fence_before();
     __syncthreads();
+#ifdef KSA_TRACE
+    if (tid == 0 && blockIdx.x < 256) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); g_cta_span[1][blockIdx.x] = t_; }
+#endif
     if (warp == kProducerWarp) tmem_dealloc(tmem, 512);
 }
 
 #ifdef KSA_TRACE
+extern "C" __attribute__((visibility("default"))) int ksa_debug_read_spans(void* spans)
+{
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(spans, g_cta_span, sizeof(g_cta_span));
+}
+
 extern "C" __attribute__((visibility("default"))) int ksa_debug_read_trace(void* ev, void* cnt, int reset)
 {
     cudaDeviceSynchronize();
