@@ -47,7 +47,7 @@ extern "C" {
 /* ---- status codes ------------------------------------------------------------------- */
 #define KSA_OK                 0
 #define KSA_ERR_INVALID_ARG   -1   /* null pointer, k < 1, m < 0, C < 0, bad lengths/strides/alignment */
-#define KSA_ERR_UNSUPPORTED   -2   /* head_dim not 64/128, device is not sm_100, limits exceeded      */
+#define KSA_ERR_UNSUPPORTED   -2   /* head_dim not 64/128, device is not sm_100, limits exceeded (more than 65,535 sequences, 1,024 query heads, 2^30 packed rows) */
 #define KSA_ERR_WORKSPACE     -3   /* workspace missing or smaller than ksa_workspace_bytes            */
 #define KSA_ERR_CUDA          -4   /* a CUDA runtime/driver call failed (see ksa_last_cuda_error)      */
 #define KSA_ERR_TIMEOUT       -5   /* a bounded device-side wait gave up (see ksa_last_device_status)  */

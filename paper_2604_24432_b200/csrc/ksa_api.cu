@@ -75,6 +75,7 @@ int validate(const ksa_params* p)
     if (p->head_dim != 64 && p->head_dim != 128) return KSA_ERR_UNSUPPORTED;
     if (p->num_q_heads > 1024 || p->chunk_len > (1 << 20) || p->summaries_per_chunk > (1 << 20))
         return KSA_ERR_UNSUPPORTED;
+    if (p->num_seqs > 65535) return KSA_ERR_UNSUPPORTED;          // sequences are a grid dimension of the helper kernels
     // padded stream rows must fit comfortably in int32
     int64_t n_total = p->cu_text_lens[p->num_seqs];
     if (n_total + (int64_t)p->num_seqs * kTileM > (1ll << 30)) return KSA_ERR_UNSUPPORTED;

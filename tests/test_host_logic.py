@@ -170,3 +170,25 @@ def test_workspace_size_formula():
     want = (8 + 2 + 2) * text_rows * 256 + 4 * summ_rows * 256
     got = ksa.workspace_bytes(prob)
     assert want <= got <= want + 5 * 1024
+
+
+def test_no_pack_mode_needs_no_workspace():
+    """Whole chunks everywhere and a tile that is a whole number of chunks: nothing is packed."""
+    assert ksa.workspace_bytes(ksa.Problem([1024, 640], 8, 1, 4, 8, 2, 128, 0.088)) == 256
+    assert ksa.workspace_bytes(ksa.Problem([1024, 640], 8, 0, 4, 8, 2, 128, 0.088)) == 256
+    assert ksa.workspace_bytes(ksa.Problem([1024, 641], 8, 1, 4, 8, 2, 128, 0.088)) > 256      # ragged tail
+    assert ksa.workspace_bytes(ksa.Problem([1020], 3, 1, 4, 8, 2, 128, 0.088)) > 256           # 128 % k != 0
+    assert ksa.workspace_bytes(ksa.Problem([1024], 8, 3, 4, 8, 2, 128, 0.088)) > 256           # 128 % m != 0
+    ref = ksa.Problem([1024, 640], 8, 1, 4, 8, 2, 128, 0.088, ksa.KSA_FLAG_REFERENCE_KERNEL)
+    assert ksa.workspace_bytes(ref) > 256                                                      # cross-check kernel reads the packed streams
+
+
+def test_backward_workspace_and_limits():
+    prob = ksa.Problem([1000, 300], 8, 1, 4, 8, 2, 128, 0.088)
+    text_rows, summ_rows = 1024 + 384, 128 + 128
+    fwd = (8 + 2 + 2) * text_rows * 256 + 4 * summ_rows * 256
+    extra = 8 * text_rows * 256 + 2 * 8 * text_rows * 4 + 2 * 2 * (text_rows + summ_rows) * 128 * 4
+    got = ksa.bwd_workspace_bytes(prob)
+    assert fwd + extra <= got <= fwd + extra + 16 * 1024
+    many = ksa.Problem([8] * 70000, 8, 1, 2, 4, 2, 64, 0.125)
+    assert _status_of(lambda: ksa.workspace_bytes(many)) == ksa.KSA_ERR_UNSUPPORTED
