@@ -742,12 +742,30 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     a.qt = fa.qt; a.kt = fa.kt; a.vt = fa.vt; a.ks = fa.ks; a.vs = fa.vs;
     a.dot = (uint16_t*)(ws + bl.dot); a.lse_t = (float*)(ws + bl.lse_t); a.delta_t = (float*)(ws + bl.delta_t);
     a.dkt = (float*)(ws + bl.dkt); a.dvt = (float*)(ws + bl.dvt); a.dks = (float*)(ws + bl.dks); a.dvs = (float*)(ws + bl.dvs);
+    a.status = ctx->d_status;
     // the four accumulators are contiguous in the workspace: one clear
     if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_dq(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if (a.D == 128) {
+        // dK / dV on the tcgen05 tensor cores, fed by TMA from the packed streams
+        static bool bwd_tc_ready = false;
+        if (!bwd_tc_ready) {
+            if ((e = setup_bwd_tc()) != cudaSuccess) return cuda_fail(ctx, e);
+            bwd_tc_ready = true;
+        }
+        BwdMaps bm;
+        if ((rc = encode_stream_map(ctx, &bm.qt, const_cast<uint16_t*>(a.qt), a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &bm.dot, a.dot, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &bm.kt, const_cast<uint16_t*>(a.kt), a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &bm.vt, const_cast<uint16_t*>(a.vt), a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &bm.ks, const_cast<uint16_t*>(a.ks), a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &bm.vs, const_cast<uint16_t*>(a.vs), a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+        if ((e = launch_bwd_dkv_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    } else {
+        if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    }
     if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 5 + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
     return KSA_OK;

@@ -1,5 +1,6 @@
 // Internal interface of the backward pass (kernel arguments and launchers).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "ksa_common.h"
@@ -25,7 +26,12 @@ struct BwdArgs {
     float* delta_t;             // [Hq][text_rows], <dO, O>
     float* dkt; float* dvt;     // [Hkv][text_rows][D] fp32
     float* dks; float* dvs;     // [Hkv][summ_rows][D] fp32
+    int32_t* status;            // device status word of the context (bounded waits report here)
 };
+
+// Tensor maps of the packed streams (boxes of 128 rows x 64 elements, 128-byte swizzle) for the
+// tensor-core kernels: Q and dO per query head, K and V of both streams per KV head.
+struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs; };
 
 // Packs the text rows of dO, lse (in log2 units) and delta = <dO, O>.
 cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream);
@@ -37,5 +43,8 @@ cudaError_t launch_bwd_dkv(const BwdArgs& a, cudaStream_t stream);
 // Accumulators -> bf16 dk / dv at the augmented positions.
 cudaError_t launch_bwd_finish(const BwdArgs& a, cudaStream_t stream);
 cudaError_t setup_bwd();
+// dK / dV on the tcgen05 tensor cores (head_dim 128 only).
+cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
+cudaError_t setup_bwd_tc();
 
 }  // namespace ksa
