@@ -531,11 +531,11 @@ extern "C" __attribute__((visibility("default"))) int ksa_schedule_dump(ksa_ctx*
 // ---------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------
-static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H)
+static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H, int box_rows = kTileN)
 {
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -747,23 +747,26 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = launch_bwd_dq(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if (a.D == 128) {
-        // dK / dV on the tcgen05 tensor cores, fed by TMA from the packed streams
+        // text rows on the tcgen05 tensor cores, fed by TMA from the packed streams
         static bool bwd_tc_ready = false;
         if (!bwd_tc_ready) {
             if ((e = setup_bwd_tc()) != cudaSuccess) return cuda_fail(ctx, e);
             bwd_tc_ready = true;
         }
         BwdMaps bm;
-        if ((rc = encode_stream_map(ctx, &bm.qt, const_cast<uint16_t*>(a.qt), a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &bm.dot, a.dot, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &bm.kt, const_cast<uint16_t*>(a.kt), a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &bm.vt, const_cast<uint16_t*>(a.vt), a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &bm.ks, const_cast<uint16_t*>(a.ks), a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
-        if ((rc = encode_stream_map(ctx, &bm.vs, const_cast<uint16_t*>(a.vs), a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+        struct { CUtensorMap* m128; CUtensorMap* m64; const void* base; int64_t rows; int H; } streams[6] = {
+            {&bm.qt, &bm.qt64, a.qt, a.text_rows, a.Hq},   {&bm.dot, &bm.dot64, a.dot, a.text_rows, a.Hq},
+            {&bm.kt, &bm.kt64, a.kt, a.text_rows, a.Hkv},  {&bm.vt, &bm.vt64, a.vt, a.text_rows, a.Hkv},
+            {&bm.ks, &bm.ks64, a.ks, a.summ_rows, a.Hkv},  {&bm.vs, &bm.vs64, a.vs, a.summ_rows, a.Hkv}};
+        for (auto& t : streams) {
+            if ((rc = encode_stream_map(ctx, t.m128, const_cast<void*>(t.base), a.D, t.rows, t.H, 128)) != KSA_OK) return rc;
+            if ((rc = encode_stream_map(ctx, t.m64, const_cast<void*>(t.base), a.D, t.rows, t.H, 64)) != KSA_OK) return rc;
+        }
+        if ((e = launch_bwd_dq_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         if ((e = launch_bwd_dkv_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     } else {
+        if ((e = launch_bwd_dq(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     }
     if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);

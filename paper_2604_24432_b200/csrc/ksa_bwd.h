@@ -29,9 +29,9 @@ struct BwdArgs {
     int32_t* status;            // device status word of the context (bounded waits report here)
 };
 
-// Tensor maps of the packed streams (boxes of 128 rows x 64 elements, 128-byte swizzle) for the
-// tensor-core kernels: Q and dO per query head, K and V of both streams per KV head.
-struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs; };
+// Tensor maps of the packed streams for the tensor-core kernels (128-byte swizzle, boxes of 64 elements x
+// 128 rows, or x 64 rows for the "64" ones): Q and dO per query head, K and V of both streams per KV head.
+struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs, qt64, dot64, kt64, vt64, ks64, vs64; };
 
 // Packs the text rows of dO, lse (in log2 units) and delta = <dO, O>.
 cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream);
@@ -43,7 +43,8 @@ cudaError_t launch_bwd_dkv(const BwdArgs& a, cudaStream_t stream);
 // Accumulators -> bf16 dk / dv at the augmented positions.
 cudaError_t launch_bwd_finish(const BwdArgs& a, cudaStream_t stream);
 cudaError_t setup_bwd();
-// dK / dV on the tcgen05 tensor cores (head_dim 128 only).
+// dQ and dK / dV of the text rows on the tcgen05 tensor cores (head_dim 128 only).
+cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
 cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
 cudaError_t setup_bwd_tc();
 

@@ -1,20 +1,28 @@
-// dK / dV of the backward pass on the sm_100a tensor cores (head_dim 128).
+// Backward pass of the text rows on the sm_100a tensor cores (head_dim 128): dK / dV and dQ.
 //
-// Key-stationary and transposed, like the mma.sync kernel it replaces for D = 128: a CTA owns one
-// tile of 128 keys of one KV head (text stream or summary stream) and walks a segment of the
-// (query tile, query head) pairs that see it.  TMEM (512 columns): ST = K Q^T [0,128),
-// DPT = V dO^T [128,256), dV [256,384), dK [384,512); lanes are the 128 keys.  Per pair:
-//   MMA     ST = K Q^T, DPT = V dO^T (shared memory x shared memory)              -> s_full
-//   warps   P^T = exp2(ST scale - lse_q) on visible pairs, dS^T = P^T (DPT - delta_q); both as
-//           bf16 over the first 16 columns of each 32-column chunk of ST / DPT    -> p_full
-//   MMA     dV += P^T dO, dK += dS^T Q (A from TMEM, B = the dO / Q tile read MN-major)
-// The Q and dO tiles stream through two shared-memory stages filled by TMA; K and V stay.
-// At the end each key row adds its dV and scale * dK to the fp32 accumulators of the stream
-// (vector atomics: several segments and the summary-row kernel add to the same rows).
-// Warps 0-7: one key row per thread, two warps per row quarter (warp w and w + 4 share the lanes
-// 32 (w % 4) ..; each takes two of the four 32-column chunks of the query tile); warp 8: TMA
-// producer; warp 9: MMA issuer.
-// Every mbarrier wait is bounded (status word + CTA-wide abort flag, as in the forward kernel).
+// Both kernels keep two 128-row operand tiles resident in shared memory, stream 64-row half
+// tiles of the other two operands through four TMA-filled slots, and run the same software
+// pipeline over "half iterations" u = 0, 1, 2, ...:
+//   MMA     X_u = A1 B1_u^T, Y_u = A2 B2_u^T   (128 x 64, shared memory x shared memory) -> s_full[u & 1]
+//   warps   P = exp2(X scale - lse) on visible pairs, dS = P (Y - delta); as bf16 over the
+//           first 16 columns of each 32-column chunk of X / Y                            -> p_full[u & 1]
+//   MMA     accumulators += (bf16 from TMEM) x (the streamed half tile read MN-major)    -> q_empty[u & 3]
+// The two TMEM buffers (u even / odd) let the products of u + 1 and the accumulations of u - 1
+// run while the warps work on u.  TMEM (512 columns): X0 [0,64) X1 [64,128) Y0 [128,192)
+// Y1 [192,256), accumulators from 256.
+//
+//   dK / dV  key-stationary and transposed: A1 = K tile, A2 = V tile (text or summary stream),
+//            B1 = Q half tile, B2 = dO half tile of the (query tile, query head) pairs that see
+//            the keys; X = S^T, Y = dP^T; dV += P^T dO, dK += dS^T Q; at the end each key row
+//            adds dV and scale * dK to the fp32 accumulators of its stream (vector atomics:
+//            several segments and the summary-row kernel add to the same rows).
+//   dQ       query-stationary: A1 = Q tile, A2 = dO tile, B1 = K half tile, B2 = V half tile over
+//            the visible summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP;
+//            dQ += dS K; at the end scale * dQ goes to the caller's tensor as bf16.
+//
+// Warps 0-7: one accumulator row per thread, two warps per row quarter (warp w and w + 4 share the
+// lanes 32 (w % 4) ..; each takes one 32-column chunk of a half tile); warp 8: TMA producer;
+// warp 9: MMA issuer.  Every mbarrier wait is bounded (status word + CTA-wide abort flag).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -27,16 +35,17 @@ namespace ksa {
 using namespace ptx;
 
 constexpr int kBwdTcThreads = 320;
-constexpr int kBwdSegTiles = 8;                 // query tiles (of 128 rows) per segment
-constexpr int kBwdTileBytes = 128 * 128 * 2;    // one 128 x 128 bf16 tile
+constexpr int kBwdSegTiles = 16;                // dK / dV: query tiles (of 128 rows) per CTA
+constexpr int kBwdTileBytes = 128 * 128 * 2;    // one 128 x 128 bf16 tile: [d half][128 rows][128 B]
+constexpr int kBwdSlotBytes = 2 * 64 * 128 * 2; // two 64 x 128 half tiles, each [d half][64 rows][128 B]
 
 // shared memory map (bytes from the 1024-aligned base)
-constexpr int kOffK = 0, kOffV = kBwdTileBytes, kOffQ = 2 * kBwdTileBytes;            // Q stage s at kOffQ + s * 2 tiles, dO right after Q
-constexpr int kOffBars = 6 * kBwdTileBytes;                                           // 8 barriers
-constexpr int kOffMisc = kOffBars + 64;                                               // TMEM slot, abort flags
-constexpr int kOffRow = kOffMisc + 64;                                                // [8 warps][3][64] per-query scalars
-constexpr int kBwdTcSmem = kOffRow + 8 * 3 * 64 * 4 + 1024;
-enum : int { BB_KVFULL = 0, BB_QFULL = 1, BB_QEMPTY = 3, BB_SFULL = 5, BB_PFULL = 6, BB_OFULL = 7 };
+constexpr int kOffA1 = 0, kOffA2 = kBwdTileBytes, kOffSlots = 2 * kBwdTileBytes;
+constexpr int kOffBars = kOffSlots + 4 * kBwdSlotBytes;                               // 14 barriers
+constexpr int kOffMisc = kOffBars + 128;                                              // TMEM slot, abort flags
+constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [8 warps][2][3][64] per-query scalars
+constexpr int kBwdTcSmem = kOffRow + 8 * 2 * 3 * 64 * 4 + 1024;
+enum : int { BB_AFULL = 0, BB_QFULL = 1, BB_QEMPTY = 5, BB_SFULL = 9, BB_PFULL = 11, BB_OFULL = 13 };
 
 __device__ __forceinline__ uint32_t bt_ld_shared(uint32_t addr)
 {
@@ -65,17 +74,125 @@ __device__ __forceinline__ bool bt_wait(uint32_t bar, uint32_t parity, uint32_t 
     }
 }
 
+// Shared-memory layout and barrier addresses of one CTA.
+struct BtSmem {
+    uint32_t base;
+    __device__ __forceinline__ uint32_t a1() const { return base + kOffA1; }
+    __device__ __forceinline__ uint32_t a2() const { return base + kOffA2; }
+    __device__ __forceinline__ uint32_t b1(int slot) const { return base + kOffSlots + (uint32_t)slot * kBwdSlotBytes; }
+    __device__ __forceinline__ uint32_t b2(int slot) const { return b1(slot) + kBwdSlotBytes / 2; }
+    __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBars + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t tmem_slot() const { return base + kOffMisc; }
+    __device__ __forceinline__ uint32_t abort_addr() const { return base + kOffMisc + 4; }
+};
+
+__device__ __forceinline__ void bt_init(const BtSmem& sm, int tid, int warp)
+{
+    if (tid == 0) {
+        mbar_init(sm.bar(BB_AFULL), 1);
+        for (int s = 0; s < 4; ++s) { mbar_init(sm.bar(BB_QFULL + s), 1); mbar_init(sm.bar(BB_QEMPTY + s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(sm.bar(BB_SFULL + s), 1); mbar_init(sm.bar(BB_PFULL + s), 8); }
+        mbar_init(sm.bar(BB_OFULL), 1);
+        bt_st_shared(sm.abort_addr(), 0u);
+        bt_st_shared(sm.abort_addr() + 4, 0u);
+        fence_mbar_init();
+    }
+    if (warp == 8) { tmem_alloc(sm.tmem_slot(), 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+}
+
+// The MMA issuer's whole loop.  kAcc = number of accumulators (2: dV from X and B2, dK from Y and B1;
+// 1: dQ from X and B1).
+template <int kAcc>
+__device__ __forceinline__ void bt_mma_loop(const BtSmem& sm, uint32_t tmem, int U, int32_t* status)
+{
+    constexpr uint32_t idesc_ss = make_idesc_bf16(128, 64, false);      // both operands K-major, N = 64
+    constexpr uint32_t idesc_ts = make_idesc_bf16(128, 128, true);      // B read MN-major, N = 128
+    const uint32_t abort_addr = sm.abort_addr();
+    const uint64_t a1d = make_smem_desc_sw128(sm.a1(), 16, 1024), a2d = make_smem_desc_sw128(sm.a2(), 16, 1024);
+    auto products = [&](int u) -> bool {
+        const int slot = u & 3, buf = u & 1;
+        if (!bt_wait(sm.bar(BB_QFULL + slot), (u >> 2) & 1, abort_addr, status, kStatusWaitQFull)) return false;
+        tc_fence_after();
+        const uint64_t b1d = make_smem_desc_sw128(sm.b1(slot), 16, 1024), b2d = make_smem_desc_sw128(sm.b2(slot), 16, 1024);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+            mma_ss(tmem + buf * 64, a1d + (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
+                   b1d + (uint32_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4), idesc_ss, kk > 0 ? 1u : 0u);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+            mma_ss(tmem + 128 + buf * 64, a2d + (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
+                   b2d + (uint32_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4), idesc_ss, kk > 0 ? 1u : 0u);
+        tc_commit(sm.bar(BB_SFULL + buf));
+        return true;
+    };
+    bool alive = bt_wait(sm.bar(BB_AFULL), 0, abort_addr, status, kStatusWaitKvFull);
+    if (alive) alive = products(0);
+    if (alive && U > 1) alive = products(1);
+    for (int u = 0; u < U && alive; ++u) {
+        const int slot = u & 3, buf = u & 1;
+        if (!bt_wait(sm.bar(BB_PFULL + buf), (u >> 1) & 1, abort_addr, status, kStatusWaitPFull)) break;
+        tc_fence_after();
+        // half tile read MN-major: 64-element atoms of d are 8192 bytes apart, 8-row groups 1024 bytes
+        const uint64_t b1m = make_smem_desc_sw128(sm.b1(slot), 8192, 1024), b2m = make_smem_desc_sw128(sm.b2(slot), 8192, 1024);
+        if (kAcc == 2) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                mma_ts(tmem + 256, tmem + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b2m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (u > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                mma_ts(tmem + 384, tmem + 128 + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (u > 0 || kk > 0) ? 1u : 0u);
+        } else {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                mma_ts(tmem + 256, tmem + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (u > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(sm.bar(BB_QEMPTY + slot));
+        if (u + 2 < U) alive = products(u + 2);
+    }
+    tc_commit(sm.bar(BB_OFULL));
+}
+
+// One TMA-filled slot: the 64 x 128 half tiles of two tensors (rows row .. row + 63 of head `head`).
+__device__ __forceinline__ void bt_load_slot(const BtSmem& sm, int slot, const CUtensorMap* m1, const CUtensorMap* m2, int row, int head)
+{
+    const uint32_t bar = sm.bar(BB_QFULL + slot);
+    mbar_arrive_expect_tx(bar, (uint32_t)kBwdSlotBytes);
+    for (int h2 = 0; h2 < 2; ++h2) {
+        tma_load_3d(sm.b1(slot) + h2 * 8192, m1, bar, h2 * 64, row, head);
+        tma_load_3d(sm.b2(slot) + h2 * 8192, m2, bar, h2 * 64, row, head);
+    }
+}
+// The two resident 128 x 128 tiles.
+__device__ __forceinline__ void bt_load_resident(const BtSmem& sm, const CUtensorMap* m1, const CUtensorMap* m2, int row, int head)
+{
+    const uint32_t bar = sm.bar(BB_AFULL);
+    mbar_arrive_expect_tx(bar, 2u * kBwdTileBytes);
+    for (int h2 = 0; h2 < 2; ++h2) {
+        tma_load_3d(sm.a1() + h2 * 16384, m1, bar, h2 * 64, row, head);
+        tma_load_3d(sm.a2() + h2 * 16384, m2, bar, h2 * 64, row, head);
+    }
+}
+// After an abort: leave no copy in flight (bounded waits on what was issued last; the second flag is never set).
+__device__ __forceinline__ void bt_drain(const BtSmem& sm, const int (&last_u)[4], int32_t* status)
+{
+    bt_wait(sm.bar(BB_AFULL), 0, sm.abort_addr() + 4, status, kStatusWaitKvFull);
+    for (int s = 0; s < 4; ++s)
+        if (last_u[s] >= 0) bt_wait(sm.bar(BB_QFULL + s), (last_u[s] >> 2) & 1, sm.abort_addr() + 4, status, kStatusWaitQFull);
+}
+
 __global__ void __launch_bounds__(kBwdTcThreads, 1)
 ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ)
 {
     extern __shared__ uint8_t bsm_raw[];
-    const uint32_t base = (smem_u32(bsm_raw) + 1023u) & ~1023u;
-    uint8_t* base_ptr = bsm_raw + (base - smem_u32(bsm_raw));
-    const uint32_t sK = base + kOffK, sV = base + kOffV;
-    auto sQ = [&](int st) -> uint32_t { return base + kOffQ + (uint32_t)st * 2u * kBwdTileBytes; };
-    auto sG = [&](int st) -> uint32_t { return sQ(st) + kBwdTileBytes; };
-    auto bar = [&](int i) -> uint32_t { return base + kOffBars + 8u * (uint32_t)i; };
-    const uint32_t tmem_slot = base + kOffMisc, abort_addr = tmem_slot + 4;
+    BtSmem sm;
+    sm.base = (smem_u32(bsm_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = bsm_raw + (sm.base - smem_u32(bsm_raw));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- which keys, which queries (Eq. 3) ------------------------------------------------------
@@ -101,165 +218,141 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     const int seg0 = qt_lo + (int)blockIdx.x * kBwdSegTiles;
     if (seg0 > qt_hi) return;
     const int seg1 = min(qt_hi + 1, seg0 + kBwdSegTiles);
-    const int iters = (seg1 - seg0) * G;
+    const int iters = (seg1 - seg0) * G;                                  // (query tile, query head) pairs
+    const int U = 2 * iters;                                              // half iterations
     const int krow0 = (summ ? sq.summ_off : sq.text_off) + kt * 128;      // first row of the tile in its packed stream
 
-    if (tid == 0) {
-        mbar_init(bar(BB_KVFULL), 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(bar(BB_QFULL + s), 1); mbar_init(bar(BB_QEMPTY + s), 1); }
-        mbar_init(bar(BB_SFULL), 1);
-        mbar_init(bar(BB_PFULL), 8);
-        mbar_init(bar(BB_OFULL), 1);
-        bt_st_shared(abort_addr, 0u);
-        bt_st_shared(abort_addr + 4, 0u);
-        fence_mbar_init();
-    }
-    if (warp == 8) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = bt_ld_shared(tmem_slot);
+    bt_init(sm, tid, warp);
+    const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
 
     if (warp == 8) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
-            prefetch_tensormap(&maps.qt); prefetch_tensormap(&maps.dot);
-            const CUtensorMap* mk = summ ? &maps.ks : &maps.kt;
-            const CUtensorMap* mv = summ ? &maps.vs : &maps.vt;
-            mbar_arrive_expect_tx(bar(BB_KVFULL), 2u * kBwdTileBytes);
-            for (int h2 = 0; h2 < 2; ++h2) {
-                tma_load_3d(sK + h2 * 16384, mk, bar(BB_KVFULL), h2 * 64, krow0, hk);
-                tma_load_3d(sV + h2 * 16384, mv, bar(BB_KVFULL), h2 * 64, krow0, hk);
-            }
-            int last_it[2] = {-1, -1};
-            for (int it = 0; it < iters; ++it) {
-                const int st = it & 1;
-                if (!bt_wait(bar(BB_QEMPTY + st), ((it >> 1) & 1) ^ 1u, abort_addr, a.status, kStatusWaitQEmpty)) break;
+            prefetch_tensormap(&maps.qt64); prefetch_tensormap(&maps.dot64);
+            bt_load_resident(sm, summ ? &maps.ks : &maps.kt, summ ? &maps.vs : &maps.vt, krow0, hk);
+            int last_u[4] = {-1, -1, -1, -1};
+            for (int u = 0; u < U; ++u) {
+                const int slot = u & 3, it = u >> 1;
+                if (!bt_wait(sm.bar(BB_QEMPTY + slot), ((u >> 2) & 1) ^ 1u, sm.abort_addr(), a.status, kStatusWaitQEmpty)) break;
                 const int qt = seg0 + it / G, h = hk * G + it % G;
-                mbar_arrive_expect_tx(bar(BB_QFULL + st), 2u * kBwdTileBytes);
-                last_it[st] = it;
-                for (int h2 = 0; h2 < 2; ++h2) {
-                    tma_load_3d(sQ(st) + h2 * 16384, &maps.qt, bar(BB_QFULL + st), h2 * 64, sq.text_off + qt * 128, h);
-                    tma_load_3d(sG(st) + h2 * 16384, &maps.dot, bar(BB_QFULL + st), h2 * 64, sq.text_off + qt * 128, h);
-                }
+                bt_load_slot(sm, slot, &maps.qt64, &maps.dot64, sq.text_off + qt * 128 + (u & 1) * 64, h);
+                last_u[slot] = u;
             }
-            if (bt_ld_shared(abort_addr) != 0u) {
-                // gave up: leave no copy in flight (bounded waits on what was issued last; the second flag is never set)
-                bt_wait(bar(BB_KVFULL), 0, abort_addr + 4, a.status, kStatusWaitKvFull);
-                for (int st = 0; st < 2; ++st)
-                    if (last_it[st] >= 0) bt_wait(bar(BB_QFULL + st), (last_it[st] >> 1) & 1, abort_addr + 4, a.status, kStatusWaitQFull);
-            }
+            if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, last_u, a.status);
         }
     } else if (warp == 9) {
         // =============================== MMA issuer =================================
-        if (lane == 0) {
-            constexpr uint32_t idesc_kmajor = make_idesc_bf16(128, 128, false);     // both operands K-major
-            constexpr uint32_t idesc_mnb = make_idesc_bf16(128, 128, true);         // B read MN-major
-            const uint64_t kd = make_smem_desc_sw128(sK, 16, 1024), vd = make_smem_desc_sw128(sV, 16, 1024);
-            bool alive = bt_wait(bar(BB_KVFULL), 0, abort_addr, a.status, kStatusWaitKvFull);
-            uint32_t pf_phase = 0;
-            for (int it = 0; it < iters && alive; ++it) {
-                const int st = it & 1;
-                if (!bt_wait(bar(BB_QFULL + st), (it >> 1) & 1, abort_addr, a.status, kStatusWaitQFull)) break;
-                tc_fence_after();
-                const uint64_t qd = make_smem_desc_sw128(sQ(st), 16, 1024), gd = make_smem_desc_sw128(sG(st), 16, 1024);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
-                    mma_ss(tmem + 0, kd + off, qd + off, idesc_kmajor, kk > 0 ? 1u : 0u);          // ST = K Q^T
-                }
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
-                    mma_ss(tmem + 128, vd + off, gd + off, idesc_kmajor, kk > 0 ? 1u : 0u);        // DPT = V dO^T
-                }
-                tc_commit(bar(BB_SFULL));
-                if (!bt_wait(bar(BB_PFULL), pf_phase, abort_addr, a.status, kStatusWaitPFull)) break;
-                pf_phase ^= 1u;
-                tc_fence_after();
-                const uint64_t gmn = make_smem_desc_sw128(sG(st), 16384, 1024), qmn = make_smem_desc_sw128(sQ(st), 16384, 1024);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)                                                       // dV += P^T dO
-                    mma_ts(tmem + 256, tmem + 0 + (kk >> 1) * 32 + (kk & 1) * 8, gmn + (uint32_t)((kk * 2048) >> 4), idesc_mnb, (it > 0 || kk > 0) ? 1u : 0u);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)                                                       // dK += dS^T Q
-                    mma_ts(tmem + 384, tmem + 128 + (kk >> 1) * 32 + (kk & 1) * 8, qmn + (uint32_t)((kk * 2048) >> 4), idesc_mnb, (it > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(bar(BB_QEMPTY + st));
-            }
-            tc_commit(bar(BB_OFULL));
-        }
+        if (lane == 0) bt_mma_loop<2>(sm, tmem, U, a.status);
     } else {
         // =============================== key rows ===================================
-        const int quarter = warp & 3, half = warp >> 2;                  // lanes 32 quarter ..; chunks half and half + 2
+        const int quarter = warp & 3, hh = warp >> 2;                    // lanes 32 quarter ..; columns 32 hh .. of each half tile
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-        const uint32_t tST = tmem + lane_sel, tDP = tmem + lane_sel + 128u;
         const int key_raw = kt * 128 + quarter * 32 + lane;
         const int key = key_raw < n_keys ? key_raw : 0x7fffffff;        // rows past the stream never match
-        float* rowf = reinterpret_cast<float*>(base_ptr + kOffRow) + warp * 3 * 64;      // this warp's lse / delta / bound
-        int* rowi = reinterpret_cast<int*>(rowf + 2 * 64);
-        uint32_t sf_phase = 0;
-        bool alive = true;
-        for (int it = 0; it < iters; ++it) {
+        const int key_first = kt * 128, key_last_pad = kt * 128 + 127;
+        // per-query scalars of this warp's columns, double-buffered by iteration: [buf][lse, delta, bound][64];
+        // entry x * 32 + j belongs to query column 64 x + 32 hh + j of the tile
+        float* rows = reinterpret_cast<float*>(base_ptr + kOffRow) + warp * 2 * 3 * 64;
+        float n_lse[2], n_dl[2];
+        int n_bnd[2];
+        auto fetch = [&](int it) {
             const int qt = seg0 + it / G, h = hk * G + it % G;
             const size_t r = (size_t)h * a.text_rows + sq.text_off + (size_t)qt * 128;
-            __syncwarp();
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int slot = e * 32 + lane;                           // slot j of pass e <-> column (half + 2 e) * 32 + j
-                const int col = (half + 2 * e) * 32 + lane, i = qt * 128 + col;
-                rowf[slot] = a.lse_t[r + col];
-                rowf[64 + slot] = a.delta_t[r + col];
+            for (int x = 0; x < 2; ++x) {
+                const int col = 64 * x + 32 * hh + lane, i = qt * 128 + col;
+                n_lse[x] = a.lse_t[r + col];
+                n_dl[x] = a.delta_t[r + col];
                 const int far = max(0, i / a.k - a.C);
-                rowi[slot] = (i >= sq.n_text) ? (summ ? 0 : 0x7fffffff) : (summ ? min(sq.n_summ, far * a.m) : far * a.k);
+                n_bnd[x] = (i >= sq.n_text) ? (summ ? 0 : 0x7fffffff) : (summ ? min(sq.n_summ, far * a.m) : far * a.k);
             }
-            __syncwarp();
-            bool ok = bt_wait(bar(BB_SFULL), sf_phase, abort_addr, a.status, kStatusWaitSFull);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { alive = false; break; }
-            sf_phase ^= 1u;
-            tc_fence_after();
+        };
+        auto stash = [&](int it) {
+            float* rb = rows + (it & 1) * 3 * 64;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int c = half + 2 * e;                               // 32-column chunk of the query tile
-                const int i0 = qt * 128 + c * 32;
-                uint32_t st_[32], dp_[32];
-                tmem_ld32(tST + c * 32, st_);
-                tmem_ld32(tDP + c * 32, dp_);
+            for (int x = 0; x < 2; ++x) {
+                rb[x * 32 + lane] = n_lse[x];
+                rb[64 + x * 32 + lane] = n_dl[x];
+                reinterpret_cast<int*>(rb)[128 + x * 32 + lane] = n_bnd[x];
+            }
+        };
+        fetch(0);
+        stash(0);
+        __syncwarp();
+        bool alive = true;
+        for (int it = 0; it < iters && alive; ++it) {
+            if (it + 1 < iters) fetch(it + 1);                            // lands while this iteration is worked on
+            const float* rowf = rows + (it & 1) * 3 * 64;
+            const int* rowi = reinterpret_cast<const int*>(rowf) + 128;
+            const int qt = seg0 + it / G;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                bool ok = bt_wait(sm.bar(BB_SFULL + x), it & 1, sm.abort_addr(), a.status, kStatusWaitSFull);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t tX = tmem + lane_sel + x * 64 + hh * 32, tY = tX + 128u;
+                const int i0 = qt * 128 + 64 * x + 32 * hh;               // first query of the chunk
+                uint32_t xs[32], ys[32];
+                tmem_ld32(tX, xs);
+                tmem_ld32(tY, ys);
+                // every pair of the chunk visible (rows past the streams drop out by themselves: zero K / V
+                // rows are discarded below, padding queries have lse = +inf)?
+                bool full;
+                if (!summ) {
+                    const int far_last = max(0, (i0 + 31) / a.k - a.C);
+                    full = key_last_pad <= i0 && far_last * a.k <= key_first;
+                } else {
+                    const int far_first = max(0, i0 / a.k - a.C);
+                    full = key_last_pad < far_first * a.m;
+                }
                 tc_wait_ld();
                 uint32_t pp[16], dd[16];
+                if (full) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 2) {
-                    float pv[2], dv[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int slot = e * 32 + j + u;
-                        const bool vis = summ ? (key < rowi[slot]) : (key <= i0 + j + u && key >= rowi[slot]);
-                        const float p = vis ? ex2_approx(fmaf(__uint_as_float(st_[j + u]), a.scale_log2, -rowf[slot])) : 0.f;
-                        pv[u] = p;
-                        dv[u] = vis ? p * (__uint_as_float(dp_[j + u]) - rowf[64 + slot]) : 0.f;
+                    for (int j = 0; j < 32; j += 2) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(xs[j]), a.scale_log2, -rowf[x * 32 + j]));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(xs[j + 1]), a.scale_log2, -rowf[x * 32 + j + 1]));
+                        pp[j >> 1] = pack_bf16x2(p0, p1);
+                        dd[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[j]) - rowf[64 + x * 32 + j]),
+                                                 p1 * (__uint_as_float(ys[j + 1]) - rowf[64 + x * 32 + j + 1]));
                     }
-                    pp[j >> 1] = pack_bf16x2(pv[0], pv[1]);
-                    dd[j >> 1] = pack_bf16x2(dv[0], dv[1]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float pv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int slot = x * 32 + j + e;
+                            const bool vis = summ ? (key < rowi[slot]) : (key <= i0 + j + e && key >= rowi[slot]);
+                            const float t = fmaf(__uint_as_float(xs[j + e]), a.scale_log2, -rowf[slot]);
+                            pv[e] = ex2_approx(vis ? t : -INFINITY);
+                        }
+                        pp[j >> 1] = pack_bf16x2(pv[0], pv[1]);
+                        dd[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(ys[j]) - rowf[64 + x * 32 + j]),
+                                                 pv[1] * (__uint_as_float(ys[j + 1]) - rowf[64 + x * 32 + j + 1]));
+                    }
                 }
                 // bf16 results over the first 16 columns of the chunk's own fp32 columns: no other warp reads those
-                tmem_st16(tST + c * 32, pp);
-                tmem_st16(tDP + c * 32, dd);
+                tmem_st16(tX, pp);
+                tmem_st16(tY, dd);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sm.bar(BB_PFULL + x));
             }
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BB_PFULL));
+            if (it + 1 < iters) { stash(it + 1); __syncwarp(); }
         }
         if (alive) {
-            bool ok = bt_wait(bar(BB_OFULL), 0, abort_addr, a.status, kStatusWaitOFull);
+            bool ok = bt_wait(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                // half 0 adds dV, half 1 adds scale * dK (tcgen05.ld is warp-collective: rows past the stream load, too)
+                // warps 0-3 add dV, warps 4-7 add scale * dK (tcgen05.ld is warp-collective: rows past the stream load, too)
                 const size_t arow = (size_t)hk * (summ ? a.summ_rows : a.text_rows) + (size_t)krow0 + quarter * 32 + lane;
-                float* acc = (half ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * 128;
-                const float mul = half ? a.scale : 1.f;
-                const uint32_t tacc = tmem + lane_sel + (half ? 384u : 256u);
+                float* acc = (hh ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * 128;
+                const float mul = hh ? a.scale : 1.f;
+                const uint32_t tacc = tmem + lane_sel + (hh ? 384u : 256u);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -281,9 +374,167 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
+__global__ void __launch_bounds__(kBwdTcThreads, 1)
+ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps)
+{
+    extern __shared__ uint8_t bsm_raw[];
+    BtSmem sm;
+    sm.base = (smem_u32(bsm_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // ---- which queries, which keys (Eq. 3) ------------------------------------------------------
+    const int h = blockIdx.y, hk = h / (a.Hq / a.Hkv);
+    const SeqInfo sq = a.seqs[blockIdx.z];
+    const int n_qt = (sq.n_text + 127) / 128;
+    if ((int)blockIdx.x >= n_qt) return;
+    const int qt = n_qt - 1 - (int)blockIdx.x;                            // long rows first
+    const int i_first = qt * 128, i_last = min(sq.n_text, i_first + 128) - 1;
+    const int far_first = max(0, i_first / a.k - a.C), far_last = max(0, i_last / a.k - a.C);
+    const int n_s = a.m > 0 ? (min(sq.n_summ, far_last * a.m) + 127) / 128 : 0;     // summary tiles seen by the last row
+    const int t_lo = (int)(((long long)far_first * a.k) / 128);                      // first text tile seen by the first row
+    const int U = 2 * (n_s + qt - t_lo + 1);
+    // half iteration u: summary tile u/2 while u/2 < n_s, then text tile t_lo + u/2 - n_s; rows 64 (u & 1) .. of it
+    auto half_of = [&](int u, bool& is_summ, int& key0) {
+        const int j = u >> 1;
+        is_summ = j < n_s;
+        key0 = (is_summ ? j : t_lo + j - n_s) * 128 + (u & 1) * 64;
+    };
+
+    bt_init(sm, tid, warp);
+    const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
+
+    if (warp == 8) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            prefetch_tensormap(&maps.kt64); prefetch_tensormap(&maps.vt64);
+            bt_load_resident(sm, &maps.qt, &maps.dot, sq.text_off + qt * 128, h);
+            int last_u[4] = {-1, -1, -1, -1};
+            for (int u = 0; u < U; ++u) {
+                const int slot = u & 3;
+                if (!bt_wait(sm.bar(BB_QEMPTY + slot), ((u >> 2) & 1) ^ 1u, sm.abort_addr(), a.status, kStatusWaitQEmpty)) break;
+                bool is_summ; int key0;
+                half_of(u, is_summ, key0);
+                if (is_summ) bt_load_slot(sm, slot, &maps.ks64, &maps.vs64, sq.summ_off + key0, hk);
+                else         bt_load_slot(sm, slot, &maps.kt64, &maps.vt64, sq.text_off + key0, hk);
+                last_u[slot] = u;
+            }
+            if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, last_u, a.status);
+        }
+    } else if (warp == 9) {
+        // =============================== MMA issuer =================================
+        if (lane == 0) bt_mma_loop<1>(sm, tmem, U, a.status);
+    } else {
+        // =============================== query rows =================================
+        const int quarter = warp & 3, hh = warp >> 2;                    // lanes 32 quarter ..; columns 32 hh .. of each half tile
+        const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+        const int i_w0 = i_first + quarter * 32, i = i_w0 + lane;         // this thread's query row
+        const size_t r = (size_t)h * a.text_rows + sq.text_off + i;
+        const float lse2 = a.lse_t[r], dl = a.delta_t[r];                 // +inf / 0 on padding rows: P = 0 there
+        const int far_i = max(0, i / a.k - a.C);
+        const int lo_i = far_i * a.k, cnt_i = min(sq.n_summ, far_i * a.m);
+        const int far_w0 = max(0, i_w0 / a.k - a.C), far_w1 = max(0, (i_w0 + 31) / a.k - a.C);
+        bool alive = true;
+        for (int u = 0; u < U; ++u) {
+            const int x = u & 1;
+            bool ok = bt_wait(sm.bar(BB_SFULL + x), (u >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitSFull);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { alive = false; break; }
+            tc_fence_after();
+            bool is_summ; int key0;
+            half_of(u, is_summ, key0);
+            const int kc0 = key0 + 32 * hh;                               // first key of this warp's chunk
+            const uint32_t tX = tmem + lane_sel + x * 64 + hh * 32, tY = tX + 128u;
+            // the warp's 32 x 32 block: all visible, none, or mixed (rows of zeros past a stream add nothing to dQ)
+            bool full, none;
+            if (is_summ) {
+                full = kc0 + 31 < min(sq.n_summ, far_w0 * a.m);
+                none = kc0 >= far_w1 * a.m;
+            } else {
+                full = kc0 + 31 <= i_w0 && far_w1 * a.k <= kc0;
+                none = kc0 > i_w0 + 31 || kc0 + 31 < far_w0 * a.k;
+            }
+            uint32_t dd[16];
+            if (none) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dd[j] = 0u;
+            } else {
+                uint32_t xs[32], ys[32];
+                tmem_ld32(tX, xs);
+                tmem_ld32(tY, ys);
+                tc_wait_ld();
+                if (full) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(xs[j]), a.scale_log2, -lse2));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(xs[j + 1]), a.scale_log2, -lse2));
+                        dd[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[j]) - dl), p1 * (__uint_as_float(ys[j + 1]) - dl));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float pv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int key = kc0 + j + e;
+                            const bool vis = is_summ ? (key < cnt_i) : (key <= i && key >= lo_i);
+                            const float t = fmaf(__uint_as_float(xs[j + e]), a.scale_log2, -lse2);
+                            pv[e] = ex2_approx(vis ? t : -INFINITY);
+                        }
+                        dd[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(ys[j]) - dl), pv[1] * (__uint_as_float(ys[j + 1]) - dl));
+                    }
+                }
+            }
+            tmem_st16(tX, dd);                                            // dS as bf16 over the chunk's own first 16 columns
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.bar(BB_PFULL + x));
+        }
+        if (alive) {
+            bool ok = bt_wait(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                // scale * dQ as bf16 to the row's augmented position (Eq. 1); warps 0-3 the first 64 elements, 4-7 the rest
+                const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * (a.k + a.m) + (i % a.k);
+                uint16_t* dst = a.dq + aug * a.dq_st + (int64_t)h * a.dq_sh + hh * 64;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem + lane_sel + 256u + hh * 64 + c * 32, o);
+                    tc_wait_ld();
+                    if (i < sq.n_text) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(o[e]) * a.scale, __uint_as_float(o[e + 1]) * a.scale);
+                            w.y = pack_bf16x2(__uint_as_float(o[e + 2]) * a.scale, __uint_as_float(o[e + 3]) * a.scale);
+                            w.z = pack_bf16x2(__uint_as_float(o[e + 4]) * a.scale, __uint_as_float(o[e + 5]) * a.scale);
+                            w.w = pack_bf16x2(__uint_as_float(o[e + 6]) * a.scale, __uint_as_float(o[e + 7]) * a.scale);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + e) = w;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
 cudaError_t setup_bwd_tc()
 {
-    return cudaFuncSetAttribute(ksa_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdTcSmem);
+    cudaError_t e = cudaFuncSetAttribute(ksa_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdTcSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(ksa_bwd_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdTcSmem);
+}
+
+cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream)
+{
+    dim3 grid((unsigned)(a.max_text_pad / 128), (unsigned)a.Hq, (unsigned)a.num_seqs);
+    ksa_bwd_dq_tc_kernel<<<grid, kBwdTcThreads, kBwdTcSmem, stream>>>(a, maps);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream)
