@@ -5,8 +5,12 @@
 // pipeline over "half iterations" u = 0, 1, 2, ...:
 //   MMA     X_u = A1 B1_u^T, Y_u = A2 B2_u^T   (128 x 64, shared memory x shared memory) -> s_full[u & 1]
 //   warps   P = exp2(X scale - lse) on visible pairs, dS = P (Y - delta); as bf16 over the
-//           first 16 columns of each 32-column chunk of X / Y                            -> p_full[u & 1]
-//   MMA     accumulators += (bf16 from TMEM) x (the streamed half tile read MN-major)    -> q_empty[u & 3]
+//           first 8 columns of each 16-column chunk of X / Y                             -> p_full[u & 1]
+//   MMA     accumulators += (bf16 from TMEM) x (the streamed half tile read MN-major)
+// The tensor pipe works in order, so s_full of u + 2 also tells the producer that slot u & 3 is free again.
+// The issuing thread pays a few hundred cycles per wait / fence / commit while the tensor pipe runs dry
+// (its queue is short), so it waits once per half iteration: row warp 0 checks the slot of u + 2 before
+// it arrives on p_full[u & 1].
 // The two TMEM buffers (u even / odd) let the products of u + 1 and the accumulations of u - 1
 // run while the warps work on u.  TMEM (512 columns): X0 [0,64) X1 [64,128) Y0 [128,192)
 // Y1 [192,256), accumulators from 256.
@@ -20,9 +24,11 @@
 //            the visible summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP;
 //            dQ += dS K; at the end scale * dQ goes to the caller's tensor as bf16.
 //
-// Warps 0-7: one accumulator row per thread, two warps per row quarter (warp w and w + 4 share the
-// lanes 32 (w % 4) ..; each takes one 32-column chunk of a half tile); warp 8: TMA producer;
-// warp 9: MMA issuer.  Every mbarrier wait is bounded (status word + CTA-wide abort flag).
+// Warps 0-15: one accumulator row per thread, four warps per row quarter (warps w, w + 4, w + 8, w + 12
+// share the lanes 32 (w % 4) ..; each takes one 16-column chunk of a half tile: the element-wise work has
+// no reduction across columns, and four warps per scheduler hide the TMEM load / store latencies);
+// warp 16: TMA producer; warp 17: MMA issuer.  Every mbarrier wait is bounded (status word + CTA-wide
+// abort flag).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -34,18 +40,33 @@ namespace ksa {
 
 using namespace ptx;
 
-constexpr int kBwdTcThreads = 320;
+constexpr int kBwdTcThreads = 576;
+constexpr int kBwdTcRegs = 96;                  // 18 warps: five on a scheduler, 5 x 32 x 96 registers fit its file
 constexpr int kBwdSegTiles = 16;                // dK / dV: query tiles (of 128 rows) per CTA
 constexpr int kBwdTileBytes = 128 * 128 * 2;    // one 128 x 128 bf16 tile: [d half][128 rows][128 B]
 constexpr int kBwdSlotBytes = 2 * 64 * 128 * 2; // two 64 x 128 half tiles, each [d half][64 rows][128 B]
 
 // shared memory map (bytes from the 1024-aligned base)
 constexpr int kOffA1 = 0, kOffA2 = kBwdTileBytes, kOffSlots = 2 * kBwdTileBytes;
-constexpr int kOffBars = kOffSlots + 4 * kBwdSlotBytes;                               // 14 barriers
+constexpr int kOffBars = kOffSlots + 4 * kBwdSlotBytes;                               // 10 barriers
 constexpr int kOffMisc = kOffBars + 128;                                              // TMEM slot, abort flags
-constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [8 warps][2][3][64] per-query scalars
-constexpr int kBwdTcSmem = kOffRow + 8 * 2 * 3 * 64 * 4 + 1024;
-enum : int { BB_AFULL = 0, BB_QFULL = 1, BB_QEMPTY = 5, BB_SFULL = 9, BB_PFULL = 11, BB_OFULL = 13 };
+constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [16 warps][2][3][32] per-query scalars
+constexpr int kBwdTcSmem = kOffRow + 16 * 2 * 3 * 32 * 4 + 1024;
+// Optional event trace (compile with -DKSA_BWD_TRACE): one CTA of the dQ kernel records (event id, clock)
+// pairs for the MMA issuer and lane 0 of every row warp; ksa_debug_read_bwd_trace() copies them out.
+#ifdef KSA_BWD_TRACE
+constexpr int kBtEvents = 4096;
+__device__ uint2 g_btrace[17][kBtEvents];         // role 0: MMA issuer; 1 + w: row warp w
+__device__ uint32_t g_btrace_cnt[17];
+#define KSA_BT(role, id)                                                                         \
+    do {                                                                                         \
+        if (bt_on && bt_n < (uint32_t)kBtEvents) g_btrace[role][bt_n++] = make_uint2((uint32_t)(id), (uint32_t)clock()); \
+    } while (0)
+#else
+#define KSA_BT(role, id) do { } while (0)
+#endif
+
+enum : int { BB_AFULL = 0, BB_QFULL = 1, BB_SFULL = 5, BB_PFULL = 7, BB_OFULL = 9 };
 
 __device__ __forceinline__ uint32_t bt_ld_shared(uint32_t addr)
 {
@@ -74,6 +95,33 @@ __device__ __forceinline__ bool bt_wait(uint32_t bar, uint32_t parity, uint32_t 
     }
 }
 
+// The MMA issuer's wait: its time is the kernel's critical path, and a try_wait costs it a few hundred cycles
+// even when the phase is already complete; test_wait returns at once, so it spins on that.
+__device__ __forceinline__ bool bt_wait_spin(uint32_t bar, uint32_t parity, uint32_t abort_addr, int32_t* status, int code)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (bt_ld_shared(abort_addr) != 0u) return false;
+            if (clock64() - t0 > (1ll << 31)) {
+                atomicCAS(status, 0, code);
+                bt_st_shared(abort_addr, 1u);
+                return false;
+            }
+        }
+    }
+}
+
+// One lane polls for the warp (512 polling threads would crowd the barrier unit and slow the MMA issuer's waits).
+__device__ __forceinline__ bool bt_wait_warp(uint32_t bar, uint32_t parity, uint32_t abort_addr, int32_t* status, int code, int lane)
+{
+    bool ok = true;
+    if (lane == 0) ok = bt_wait(bar, parity, abort_addr, status, code);
+    return __shfl_sync(0xffffffffu, ok, 0);
+}
+
 // Shared-memory layout and barrier addresses of one CTA.
 struct BtSmem {
     uint32_t base;
@@ -90,32 +138,43 @@ __device__ __forceinline__ void bt_init(const BtSmem& sm, int tid, int warp)
 {
     if (tid == 0) {
         mbar_init(sm.bar(BB_AFULL), 1);
-        for (int s = 0; s < 4; ++s) { mbar_init(sm.bar(BB_QFULL + s), 1); mbar_init(sm.bar(BB_QEMPTY + s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(sm.bar(BB_SFULL + s), 1); mbar_init(sm.bar(BB_PFULL + s), 8); }
+        for (int s = 0; s < 4; ++s) mbar_init(sm.bar(BB_QFULL + s), 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(sm.bar(BB_SFULL + s), 1); mbar_init(sm.bar(BB_PFULL + s), 16); }
         mbar_init(sm.bar(BB_OFULL), 1);
         bt_st_shared(sm.abort_addr(), 0u);
         bt_st_shared(sm.abort_addr() + 4, 0u);
         fence_mbar_init();
     }
-    if (warp == 8) { tmem_alloc(sm.tmem_slot(), 512); tmem_relinquish(); }
+    if (warp == 16) { tmem_alloc(sm.tmem_slot(), 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 }
 
-// The MMA issuer's whole loop.  kAcc = number of accumulators (2: dV from X and B2, dK from Y and B1;
-// 1: dQ from X and B1).
+// One MMA issuer's whole loop: the half iterations u = par, par + step, ...  kAcc = number of accumulators
+// (2: dV from X and B2 at acc_col, dK from Y and B1 at acc_col + 128; 1: dQ from X and B1 at acc_col).
+// acc_zeroed: the accumulators were cleared beforehand (issuers that share them cannot tell who is first).
 template <int kAcc>
-__device__ __forceinline__ void bt_mma_loop(const BtSmem& sm, uint32_t tmem, int U, int32_t* status)
+__device__ __forceinline__ void bt_mma_loop(const BtSmem& sm, uint32_t tmem, int U, int32_t* status, int par, int step,
+                                            uint32_t acc_col, bool acc_zeroed, bool bt_on = false)
 {
+    uint32_t bt_n = 0;
+    (void)bt_on; (void)bt_n;
+#if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 2
+    uint32_t bt_wait_sum = 0;
+    const uint32_t bt_t_begin = (uint32_t)clock();
+    const bool bt_sum_on = bt_on;
+    bt_on = false;
+#endif
     constexpr uint32_t idesc_ss = make_idesc_bf16(128, 64, false);      // both operands K-major, N = 64
     constexpr uint32_t idesc_ts = make_idesc_bf16(128, 128, true);      // B read MN-major, N = 128
     const uint32_t abort_addr = sm.abort_addr();
     const uint64_t a1d = make_smem_desc_sw128(sm.a1(), 16, 1024), a2d = make_smem_desc_sw128(sm.a2(), 16, 1024);
-    auto products = [&](int u) -> bool {
+    // wait_slot: only for the first ones; later slots were checked by row warp 0 before its p_full arrival
+    auto products = [&](int u, bool wait_slot) -> bool {
         const int slot = u & 3, buf = u & 1;
-        if (!bt_wait(sm.bar(BB_QFULL + slot), (u >> 2) & 1, abort_addr, status, kStatusWaitQFull)) return false;
-        tc_fence_after();
+        if (wait_slot && !bt_wait(sm.bar(BB_QFULL + slot), (u >> 2) & 1, abort_addr, status, kStatusWaitQFull)) return false;
+        KSA_BT(0, 5);
         const uint64_t b1d = make_smem_desc_sw128(sm.b1(slot), 16, 1024), b2d = make_smem_desc_sw128(sm.b2(slot), 16, 1024);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
@@ -125,37 +184,67 @@ __device__ __forceinline__ void bt_mma_loop(const BtSmem& sm, uint32_t tmem, int
         for (int kk = 0; kk < 8; ++kk)
             mma_ss(tmem + 128 + buf * 64, a2d + (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
                    b2d + (uint32_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4), idesc_ss, kk > 0 ? 1u : 0u);
+        KSA_BT(0, 6);
         tc_commit(sm.bar(BB_SFULL + buf));
+        KSA_BT(0, 4);
+#ifdef KSA_BWD_TRACE
+        if (bt_on) { const uint32_t probe = bt_ld_shared(sm.abort_addr() + 4); if (probe == 12345u) bt_n = 0; KSA_BT(0, 30); }
+#endif
         return true;
     };
     bool alive = bt_wait(sm.bar(BB_AFULL), 0, abort_addr, status, kStatusWaitKvFull);
-    if (alive) alive = products(0);
-    if (alive && U > 1) alive = products(1);
-    for (int u = 0; u < U && alive; ++u) {
+    if (alive) alive = products(par, true);
+    if (alive && step == 1 && U > 1) alive = products(1, true);
+    for (int u = par; u < U && alive; u += step) {
         const int slot = u & 3, buf = u & 1;
-        if (!bt_wait(sm.bar(BB_PFULL + buf), (u >> 1) & 1, abort_addr, status, kStatusWaitPFull)) break;
+#if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 2
+        const uint32_t tw0 = (uint32_t)clock();
+#endif
+        if (!bt_wait_spin(sm.bar(BB_PFULL + buf), (u >> 1) & 1, abort_addr, status, kStatusWaitPFull)) break;
+#if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 2
+        bt_wait_sum += (uint32_t)clock() - tw0;
+#endif
+        KSA_BT(0, 1);
         tc_fence_after();
+        KSA_BT(0, 7);
         // half tile read MN-major: 64-element atoms of d are 8192 bytes apart, 8-row groups 1024 bytes
         const uint64_t b1m = make_smem_desc_sw128(sm.b1(slot), 8192, 1024), b2m = make_smem_desc_sw128(sm.b2(slot), 8192, 1024);
+        const bool later = acc_zeroed || u > par;
         if (kAcc == 2) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                mma_ts(tmem + 256, tmem + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b2m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
-                       (u > 0 || kk > 0) ? 1u : 0u);
+                mma_ts(tmem + acc_col, tmem + buf * 64 + kk * 16, b2m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (later || kk > 0) ? 1u : 0u);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                mma_ts(tmem + 384, tmem + 128 + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
-                       (u > 0 || kk > 0) ? 1u : 0u);
+                mma_ts(tmem + acc_col + 128, tmem + 128 + buf * 64 + kk * 16, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (later || kk > 0) ? 1u : 0u);
         } else {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                mma_ts(tmem + 256, tmem + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
-                       (u > 0 || kk > 0) ? 1u : 0u);
+                mma_ts(tmem + acc_col, tmem + buf * 64 + kk * 16, b1m + (uint32_t)((kk * 2048) >> 4), idesc_ts,
+                       (later || kk > 0) ? 1u : 0u);
         }
-        tc_commit(sm.bar(BB_QEMPTY + slot));
-        if (u + 2 < U) alive = products(u + 2);
+        KSA_BT(0, 2);
+        if (u + 2 < U) alive = products(u + 2, false);
     }
     tc_commit(sm.bar(BB_OFULL));
+#ifdef KSA_BWD_TRACE
+    if (bt_on) g_btrace_cnt[0] = bt_n;
+#if KSA_BWD_TRACE == 2
+    if (bt_sum_on) { g_btrace[0][0] = make_uint2(bt_wait_sum, (uint32_t)clock() - bt_t_begin); g_btrace[0][1] = make_uint2((uint32_t)U, 0u); g_btrace_cnt[0] = 2; }
+#endif
+#endif
+}
+
+// Producer: slot u & 3 was last read by the accumulations of u - 4, and the products of u - 2 were issued after
+// those, so their s_full completion frees the slot.  A parity wait only tells neighbouring phases apart:
+// the first time round (u = 4, 5) the phase before is waited for as well.
+__device__ __forceinline__ bool bt_slot_free(const BtSmem& sm, int u, int32_t* status)
+{
+    const uint32_t bar = sm.bar(BB_SFULL + (u & 1));
+    if (u < 6 && !bt_wait(bar, 0, sm.abort_addr(), status, kStatusWaitQEmpty)) return false;
+    return bt_wait(bar, ((u - 2) >> 1) & 1, sm.abort_addr(), status, kStatusWaitQEmpty);
 }
 
 // One TMA-filled slot: the 64 x 128 half tiles of two tensors (rows row .. row + 63 of head `head`).
@@ -186,7 +275,7 @@ __device__ __forceinline__ void bt_drain(const BtSmem& sm, const int (&last_u)[4
         if (last_u[s] >= 0) bt_wait(sm.bar(BB_QFULL + s), (last_u[s] >> 2) & 1, sm.abort_addr() + 4, status, kStatusWaitQFull);
 }
 
-__global__ void __launch_bounds__(kBwdTcThreads, 1)
+__global__ void __maxnreg__(kBwdTcRegs)
 ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ)
 {
     extern __shared__ uint8_t bsm_raw[];
@@ -225,7 +314,7 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     bt_init(sm, tid, warp);
     const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
 
-    if (warp == 8) {
+    if (warp == 16) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
             prefetch_tensormap(&maps.qt64); prefetch_tensormap(&maps.dot64);
@@ -233,48 +322,43 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             int last_u[4] = {-1, -1, -1, -1};
             for (int u = 0; u < U; ++u) {
                 const int slot = u & 3, it = u >> 1;
-                if (!bt_wait(sm.bar(BB_QEMPTY + slot), ((u >> 2) & 1) ^ 1u, sm.abort_addr(), a.status, kStatusWaitQEmpty)) break;
+                if (u >= 4 && !bt_slot_free(sm, u, a.status)) break;
                 const int qt = seg0 + it / G, h = hk * G + it % G;
                 bt_load_slot(sm, slot, &maps.qt64, &maps.dot64, sq.text_off + qt * 128 + (u & 1) * 64, h);
                 last_u[slot] = u;
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, last_u, a.status);
         }
-    } else if (warp == 9) {
+    } else if (warp == 17) {
         // =============================== MMA issuer =================================
-        if (lane == 0) bt_mma_loop<2>(sm, tmem, U, a.status);
+        if (lane == 0) bt_mma_loop<2>(sm, tmem, U, a.status, 0, 1, 256u, false);
     } else {
         // =============================== key rows ===================================
-        const int quarter = warp & 3, hh = warp >> 2;                    // lanes 32 quarter ..; columns 32 hh .. of each half tile
+        const int quarter = warp & 3, cc = warp >> 2;                    // lanes 32 quarter ..; columns 16 cc .. of each half tile
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
         const int key_raw = kt * 128 + quarter * 32 + lane;
         const int key = key_raw < n_keys ? key_raw : 0x7fffffff;        // rows past the stream never match
         const int key_first = kt * 128, key_last_pad = kt * 128 + 127;
-        // per-query scalars of this warp's columns, double-buffered by iteration: [buf][lse, delta, bound][64];
-        // entry x * 32 + j belongs to query column 64 x + 32 hh + j of the tile
-        float* rows = reinterpret_cast<float*>(base_ptr + kOffRow) + warp * 2 * 3 * 64;
-        float n_lse[2], n_dl[2];
-        int n_bnd[2];
+        // per-query scalars of this warp's columns, double-buffered by iteration: [buf][lse, delta, bound][32];
+        // entry x * 16 + j belongs to query column 64 x + 16 cc + j of the tile
+        float* rows = reinterpret_cast<float*>(base_ptr + kOffRow) + warp * 2 * 3 * 32;
+        const int my_col = 64 * (lane >> 4) + 16 * cc + (lane & 15);     // the column whose scalars this lane fetches
+        float n_lse, n_dl;
+        int n_bnd;
         auto fetch = [&](int it) {
             const int qt = seg0 + it / G, h = hk * G + it % G;
-            const size_t r = (size_t)h * a.text_rows + sq.text_off + (size_t)qt * 128;
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const int col = 64 * x + 32 * hh + lane, i = qt * 128 + col;
-                n_lse[x] = a.lse_t[r + col];
-                n_dl[x] = a.delta_t[r + col];
-                const int far = max(0, i / a.k - a.C);
-                n_bnd[x] = (i >= sq.n_text) ? (summ ? 0 : 0x7fffffff) : (summ ? min(sq.n_summ, far * a.m) : far * a.k);
-            }
+            const size_t r = (size_t)h * a.text_rows + sq.text_off + (size_t)qt * 128 + my_col;
+            const int i = qt * 128 + my_col;
+            n_lse = a.lse_t[r];
+            n_dl = a.delta_t[r];
+            const int far = max(0, i / a.k - a.C);
+            n_bnd = (i >= sq.n_text) ? (summ ? 0 : 0x7fffffff) : (summ ? min(sq.n_summ, far * a.m) : far * a.k);
         };
         auto stash = [&](int it) {
-            float* rb = rows + (it & 1) * 3 * 64;
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                rb[x * 32 + lane] = n_lse[x];
-                rb[64 + x * 32 + lane] = n_dl[x];
-                reinterpret_cast<int*>(rb)[128 + x * 32 + lane] = n_bnd[x];
-            }
+            float* rb = rows + (it & 1) * 3 * 32;
+            rb[lane] = n_lse;
+            rb[32 + lane] = n_dl;
+            reinterpret_cast<int*>(rb)[64 + lane] = n_bnd;
         };
         fetch(0);
         stash(0);
@@ -282,79 +366,82 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         bool alive = true;
         for (int it = 0; it < iters && alive; ++it) {
             if (it + 1 < iters) fetch(it + 1);                            // lands while this iteration is worked on
-            const float* rowf = rows + (it & 1) * 3 * 64;
-            const int* rowi = reinterpret_cast<const int*>(rowf) + 128;
+            const float* rowf = rows + (it & 1) * 3 * 32;
+            const int* rowi = reinterpret_cast<const int*>(rowf) + 64;
             const int qt = seg0 + it / G;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
-                bool ok = bt_wait(sm.bar(BB_SFULL + x), it & 1, sm.abort_addr(), a.status, kStatusWaitSFull);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) { alive = false; break; }
+                if (!bt_wait_warp(sm.bar(BB_SFULL + x), it & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
                 tc_fence_after();
-                const uint32_t tX = tmem + lane_sel + x * 64 + hh * 32, tY = tX + 128u;
-                const int i0 = qt * 128 + 64 * x + 32 * hh;               // first query of the chunk
-                uint32_t xs[32], ys[32];
-                tmem_ld32(tX, xs);
-                tmem_ld32(tY, ys);
+                const uint32_t tX = tmem + lane_sel + x * 64 + cc * 16, tY = tX + 128u;
+                const int i0 = qt * 128 + 64 * x + 16 * cc;               // first query of the chunk
+                uint32_t xs[16], ys[16];
+                tmem_ld16(tX, xs);
+                tmem_ld16(tY, ys);
                 // every pair of the chunk visible (rows past the streams drop out by themselves: zero K / V
                 // rows are discarded below, padding queries have lse = +inf)?
                 bool full;
                 if (!summ) {
-                    const int far_last = max(0, (i0 + 31) / a.k - a.C);
+                    const int far_last = max(0, (i0 + 15) / a.k - a.C);
                     full = key_last_pad <= i0 && far_last * a.k <= key_first;
                 } else {
                     const int far_first = max(0, i0 / a.k - a.C);
                     full = key_last_pad < far_first * a.m;
                 }
                 tc_wait_ld();
-                uint32_t pp[16], dd[16];
+                uint32_t pp[8], dd[8];
                 if (full) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(xs[j]), a.scale_log2, -rowf[x * 32 + j]));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(xs[j + 1]), a.scale_log2, -rowf[x * 32 + j + 1]));
+                    for (int j = 0; j < 16; j += 2) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(xs[j]), a.scale_log2, -rowf[x * 16 + j]));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(xs[j + 1]), a.scale_log2, -rowf[x * 16 + j + 1]));
                         pp[j >> 1] = pack_bf16x2(p0, p1);
-                        dd[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[j]) - rowf[64 + x * 32 + j]),
-                                                 p1 * (__uint_as_float(ys[j + 1]) - rowf[64 + x * 32 + j + 1]));
+                        dd[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[j]) - rowf[32 + x * 16 + j]),
+                                                 p1 * (__uint_as_float(ys[j + 1]) - rowf[32 + x * 16 + j + 1]));
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
+                    for (int j = 0; j < 16; j += 2) {
                         float pv[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int slot = x * 32 + j + e;
+                            const int slot = x * 16 + j + e;
                             const bool vis = summ ? (key < rowi[slot]) : (key <= i0 + j + e && key >= rowi[slot]);
                             const float t = fmaf(__uint_as_float(xs[j + e]), a.scale_log2, -rowf[slot]);
                             pv[e] = ex2_approx(vis ? t : -INFINITY);
                         }
                         pp[j >> 1] = pack_bf16x2(pv[0], pv[1]);
-                        dd[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(ys[j]) - rowf[64 + x * 32 + j]),
-                                                 pv[1] * (__uint_as_float(ys[j + 1]) - rowf[64 + x * 32 + j + 1]));
+                        dd[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(ys[j]) - rowf[32 + x * 16 + j]),
+                                                 pv[1] * (__uint_as_float(ys[j + 1]) - rowf[32 + x * 16 + j + 1]));
                     }
                 }
-                // bf16 results over the first 16 columns of the chunk's own fp32 columns: no other warp reads those
-                tmem_st16(tX, pp);
-                tmem_st16(tY, dd);
+                // bf16 results over the first 8 columns of the chunk's own fp32 columns: no other warp reads those
+                tmem_st8(tX, pp);
+                tmem_st8(tY, dd);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(sm.bar(BB_PFULL + x));
+                if (lane == 0) {
+                    const int u2 = 2 * it + x + 2;                        // warp 0 vouches for the slot of u + 2
+                    if (warp == 0 && u2 < U) bt_wait(sm.bar(BB_QFULL + (u2 & 3)), (u2 >> 2) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
+                    mbar_arrive(sm.bar(BB_PFULL + x));
+                }
             }
             if (it + 1 < iters) { stash(it + 1); __syncwarp(); }
         }
         if (alive) {
-            bool ok = bt_wait(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
+            if (bt_wait_warp(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull, lane)) {
                 tc_fence_after();
-                // warps 0-3 add dV, warps 4-7 add scale * dK (tcgen05.ld is warp-collective: rows past the stream load, too)
+                // odd cc: scale * dK, even cc: dV; cc / 2 picks the 64-element half of the row
+                // (tcgen05.ld is warp-collective: rows past the stream load, too)
+                const bool is_dk = (cc & 1) != 0;
+                const int d0 = (cc >> 1) * 64;
                 const size_t arow = (size_t)hk * (summ ? a.summ_rows : a.text_rows) + (size_t)krow0 + quarter * 32 + lane;
-                float* acc = (hh ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * 128;
-                const float mul = hh ? a.scale : 1.f;
-                const uint32_t tacc = tmem + lane_sel + (hh ? 384u : 256u);
+                float* acc = (is_dk ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * 128 + d0;
+                const float mul = is_dk ? a.scale : 1.f;
+                const uint32_t tacc = tmem + lane_sel + (is_dk ? 384u : 256u) + d0;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tacc + c * 32, o);
                     tc_wait_ld();
@@ -371,10 +458,10 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (warp == 16) tmem_dealloc(tmem, 512);
 }
 
-__global__ void __launch_bounds__(kBwdTcThreads, 1)
+__global__ void __maxnreg__(kBwdTcRegs)
 ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps)
 {
     extern __shared__ uint8_t bsm_raw[];
@@ -403,7 +490,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
     bt_init(sm, tid, warp);
     const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
 
-    if (warp == 8) {
+    if (warp == 16) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
             prefetch_tensormap(&maps.kt64); prefetch_tensormap(&maps.vt64);
@@ -411,7 +498,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             int last_u[4] = {-1, -1, -1, -1};
             for (int u = 0; u < U; ++u) {
                 const int slot = u & 3;
-                if (!bt_wait(sm.bar(BB_QEMPTY + slot), ((u >> 2) & 1) ^ 1u, sm.abort_addr(), a.status, kStatusWaitQEmpty)) break;
+                if (u >= 4 && !bt_slot_free(sm, u, a.status)) break;
                 bool is_summ; int key0;
                 half_of(u, is_summ, key0);
                 if (is_summ) bt_load_slot(sm, slot, &maps.ks64, &maps.vs64, sq.summ_off + key0, hk);
@@ -420,12 +507,16 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, last_u, a.status);
         }
-    } else if (warp == 9) {
+    } else if (warp == 17) {
         // =============================== MMA issuer =================================
-        if (lane == 0) bt_mma_loop<1>(sm, tmem, U, a.status);
+#ifdef KSA_BWD_TRACE
+        if (lane == 0) bt_mma_loop<1>(sm, tmem, U, a.status, 0, 1, 256u, false, blockIdx.x == 8 && blockIdx.y == 0 && blockIdx.z == 0);
+#else
+        if (lane == 0) bt_mma_loop<1>(sm, tmem, U, a.status, 0, 1, 256u, false);
+#endif
     } else {
         // =============================== query rows =================================
-        const int quarter = warp & 3, hh = warp >> 2;                    // lanes 32 quarter ..; columns 32 hh .. of each half tile
+        const int quarter = warp & 3, cc = warp >> 2;                    // lanes 32 quarter ..; columns 16 cc .. of each half tile
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
         const int i_w0 = i_first + quarter * 32, i = i_w0 + lane;         // this thread's query row
         const size_t r = (size_t)h * a.text_rows + sq.text_off + i;
@@ -434,44 +525,49 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         const int lo_i = far_i * a.k, cnt_i = min(sq.n_summ, far_i * a.m);
         const int far_w0 = max(0, i_w0 / a.k - a.C), far_w1 = max(0, (i_w0 + 31) / a.k - a.C);
         bool alive = true;
+#ifdef KSA_BWD_TRACE
+        const bool bt_on = blockIdx.x == 8 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0;
+        const int bt_role = 1 + warp;
+        uint32_t bt_n = 0;
+#endif
         for (int u = 0; u < U; ++u) {
             const int x = u & 1;
-            bool ok = bt_wait(sm.bar(BB_SFULL + x), (u >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitSFull);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { alive = false; break; }
+            if (!bt_wait_warp(sm.bar(BB_SFULL + x), (u >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
+            KSA_BT(bt_role, 10);
             tc_fence_after();
             bool is_summ; int key0;
             half_of(u, is_summ, key0);
-            const int kc0 = key0 + 32 * hh;                               // first key of this warp's chunk
-            const uint32_t tX = tmem + lane_sel + x * 64 + hh * 32, tY = tX + 128u;
-            // the warp's 32 x 32 block: all visible, none, or mixed (rows of zeros past a stream add nothing to dQ)
+            const int kc0 = key0 + 16 * cc;                               // first key of this warp's chunk
+            const uint32_t tX = tmem + lane_sel + x * 64 + cc * 16, tY = tX + 128u;
+            // the warp's 32 x 16 block: all visible, none, or mixed (rows of zeros past a stream add nothing to dQ)
             bool full, none;
             if (is_summ) {
-                full = kc0 + 31 < min(sq.n_summ, far_w0 * a.m);
+                full = kc0 + 15 < min(sq.n_summ, far_w0 * a.m);
                 none = kc0 >= far_w1 * a.m;
             } else {
-                full = kc0 + 31 <= i_w0 && far_w1 * a.k <= kc0;
-                none = kc0 > i_w0 + 31 || kc0 + 31 < far_w0 * a.k;
+                full = kc0 + 15 <= i_w0 && far_w1 * a.k <= kc0;
+                none = kc0 > i_w0 + 31 || kc0 + 15 < far_w0 * a.k;
             }
-            uint32_t dd[16];
+            uint32_t dd[8];
             if (none) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) dd[j] = 0u;
+                for (int j = 0; j < 8; ++j) dd[j] = 0u;
             } else {
-                uint32_t xs[32], ys[32];
-                tmem_ld32(tX, xs);
-                tmem_ld32(tY, ys);
+                uint32_t xs[16], ys[16];
+                tmem_ld16(tX, xs);
+                tmem_ld16(tY, ys);
                 tc_wait_ld();
+                KSA_BT(bt_role, 11);
                 if (full) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
+                    for (int j = 0; j < 16; j += 2) {
                         const float p0 = ex2_approx(fmaf(__uint_as_float(xs[j]), a.scale_log2, -lse2));
                         const float p1 = ex2_approx(fmaf(__uint_as_float(xs[j + 1]), a.scale_log2, -lse2));
                         dd[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[j]) - dl), p1 * (__uint_as_float(ys[j + 1]) - dl));
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
+                    for (int j = 0; j < 16; j += 2) {
                         float pv[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
@@ -484,35 +580,42 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
                     }
                 }
             }
-            tmem_st16(tX, dd);                                            // dS as bf16 over the chunk's own first 16 columns
+            KSA_BT(bt_role, 12);
+            tmem_st8(tX, dd);                                             // dS as bf16 over the chunk's own first 8 columns
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(sm.bar(BB_PFULL + x));
+            if (lane == 0) {
+                const int u2 = u + 2;                                     // warp 0 vouches for the slot of u + 2
+                if (warp == 0 && u2 < U) bt_wait(sm.bar(BB_QFULL + (u2 & 3)), (u2 >> 2) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
+                mbar_arrive(sm.bar(BB_PFULL + x));
+            }
+            KSA_BT(bt_role, 13);
         }
+#ifdef KSA_BWD_TRACE
+        if (bt_on) g_btrace_cnt[bt_role] = bt_n;
+#endif
         if (alive) {
-            bool ok = bt_wait(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
+            if (bt_wait_warp(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull, lane)) {
                 tc_fence_after();
-                // scale * dQ as bf16 to the row's augmented position (Eq. 1); warps 0-3 the first 64 elements, 4-7 the rest
+                // scale * dQ as bf16 to the row's augmented position (Eq. 1); warp group cc writes elements 32 cc ..
                 const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * (a.k + a.m) + (i % a.k);
-                uint16_t* dst = a.dq + aug * a.dq_st + (int64_t)h * a.dq_sh + hh * 64;
+                uint16_t* dst = a.dq + aug * a.dq_st + (int64_t)h * a.dq_sh + cc * 32;
+                uint32_t o0[32];
+                tmem_ld32(tmem + lane_sel + 256u + cc * 32, o0);
+                tc_wait_ld();
+                if (i < sq.n_text) {
+                    float o[32];
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tmem + lane_sel + 256u + hh * 64 + c * 32, o);
-                    tc_wait_ld();
-                    if (i < sq.n_text) {
+                    for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(o0[e]) * a.scale;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[e]) * a.scale, __uint_as_float(o[e + 1]) * a.scale);
-                            w.y = pack_bf16x2(__uint_as_float(o[e + 2]) * a.scale, __uint_as_float(o[e + 3]) * a.scale);
-                            w.z = pack_bf16x2(__uint_as_float(o[e + 4]) * a.scale, __uint_as_float(o[e + 5]) * a.scale);
-                            w.w = pack_bf16x2(__uint_as_float(o[e + 6]) * a.scale, __uint_as_float(o[e + 7]) * a.scale);
-                            *reinterpret_cast<uint4*>(dst + c * 32 + e) = w;
-                        }
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(o[e], o[e + 1]);
+                        w.y = pack_bf16x2(o[e + 2], o[e + 3]);
+                        w.z = pack_bf16x2(o[e + 4], o[e + 5]);
+                        w.w = pack_bf16x2(o[e + 6], o[e + 7]);
+                        *reinterpret_cast<uint4*>(dst + e) = w;
                     }
                 }
             }
@@ -520,8 +623,18 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (warp == 16) tmem_dealloc(tmem, 512);
 }
+
+#ifdef KSA_BWD_TRACE
+extern "C" __attribute__((visibility("default"))) int ksa_debug_read_bwd_trace(void* events, void* counts)
+{
+    cudaDeviceSynchronize();
+    cudaError_t e = cudaMemcpyFromSymbol(events, g_btrace, sizeof(g_btrace));
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(counts, g_btrace_cnt, sizeof(g_btrace_cnt));
+    return (int)e;
+}
+#endif
 
 cudaError_t setup_bwd_tc()
 {

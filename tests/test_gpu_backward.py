@@ -40,6 +40,8 @@ def _check(name, got, ref):
     ([450], 8, 1, 3, 4, 1, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
     ([1], 8, 1, 2, 2, 2, 64, 0),
     ([2100, 640], 8, 1, 16, 8, 2, 128, 0),            # several query segments per summary key tile
+    ([2500], 64, 8, 4, 4, 2, 128, 0),                 # long chunks with 8 summaries each
+    ([600, 9], 8, 1, 0, 4, 2, 128, 0),                # no window beyond the own chunk
 ])
 def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
