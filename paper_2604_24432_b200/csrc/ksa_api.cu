@@ -531,11 +531,11 @@ extern "C" __attribute__((visibility("default"))) int ksa_schedule_dump(ksa_ctx*
 // ---------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------
-static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H, int box_rows = kTileN)
+static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H)
 {
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -755,14 +755,12 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
             bwd_tc_ready = true;
         }
         BwdMaps bm;
-        struct { CUtensorMap* m128; CUtensorMap* m64; const void* base; int64_t rows; int H; } streams[6] = {
-            {&bm.qt, &bm.qt64, a.qt, a.text_rows, a.Hq},   {&bm.dot, &bm.dot64, a.dot, a.text_rows, a.Hq},
-            {&bm.kt, &bm.kt64, a.kt, a.text_rows, a.Hkv},  {&bm.vt, &bm.vt64, a.vt, a.text_rows, a.Hkv},
-            {&bm.ks, &bm.ks64, a.ks, a.summ_rows, a.Hkv},  {&bm.vs, &bm.vs64, a.vs, a.summ_rows, a.Hkv}};
-        for (auto& t : streams) {
-            if ((rc = encode_stream_map(ctx, t.m128, const_cast<void*>(t.base), a.D, t.rows, t.H, 128)) != KSA_OK) return rc;
-            if ((rc = encode_stream_map(ctx, t.m64, const_cast<void*>(t.base), a.D, t.rows, t.H, 64)) != KSA_OK) return rc;
-        }
+        struct { CUtensorMap* map; const void* base; int64_t rows; int H; } streams[6] = {
+            {&bm.qt, a.qt, a.text_rows, a.Hq},   {&bm.dot, a.dot, a.text_rows, a.Hq},
+            {&bm.kt, a.kt, a.text_rows, a.Hkv},  {&bm.vt, a.vt, a.text_rows, a.Hkv},
+            {&bm.ks, a.ks, a.summ_rows, a.Hkv},  {&bm.vs, a.vs, a.summ_rows, a.Hkv}};
+        for (auto& t : streams)
+            if ((rc = encode_stream_map(ctx, t.map, const_cast<void*>(t.base), a.D, t.rows, t.H)) != KSA_OK) return rc;
         if ((e = launch_bwd_dq_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         if ((e = launch_bwd_dkv_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     } else {

@@ -30,8 +30,8 @@ struct BwdArgs {
 };
 
 // Tensor maps of the packed streams for the tensor-core kernels (128-byte swizzle, boxes of 64 elements x
-// 128 rows, or x 64 rows for the "64" ones): Q and dO per query head, K and V of both streams per KV head.
-struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs, qt64, dot64, kt64, vt64, ks64, vs64; };
+// 128 rows): Q and dO per query head, K and V of both streams per KV head.
+struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs; };
 
 // Packs the text rows of dO, lse (in log2 units) and delta = <dO, O>.
 cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream);

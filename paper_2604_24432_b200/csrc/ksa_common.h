@@ -72,6 +72,7 @@ enum DeviceStatus : int32_t {
     kStatusOk = 0,
     kStatusWaitQFull = 1, kStatusWaitQEmpty = 2, kStatusWaitKvFull = 3, kStatusWaitKvEmpty = 4,
     kStatusWaitSFull = 5, kStatusWaitPFull = 6, kStatusWaitOFull = 7, kStatusWaitTest = 8,
+    kStatusSmemLayout = 9,      // the dynamic shared memory window did not hold the 1024-byte aligned layout
 };
 
 }  // namespace ksa
