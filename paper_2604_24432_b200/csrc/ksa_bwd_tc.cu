@@ -17,8 +17,10 @@
 //            accumulators of its stream (vector atomics: several segments and the summary-row kernel
 //            add to the same rows).
 //   dQ       query-stationary: A1 = Q tile, A2 = dO tile, B1 = K tile, B2 = V tile over the visible
-//            summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP.  Pipe order per j:
-//            X_{j+1}, dQ += dS K_j, Y_{j+1}.  At the end scale * dQ goes to the caller's tensor as bf16.
+//            summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP.  One accumulator leaves
+//            room for a second Y buffer (columns from 384), so both products of tile j + 1 are issued
+//            as soon as the warps have read X_j, and the warps never wait for the pipe: order per j:
+//            X_{j+1}, Y_{j+1}, dQ += dS K_j.  At the end scale * dQ goes to the caller's tensor as bf16.
 //
 // Warps 0-15: one accumulator row per thread, four warps per row quarter (warps w, w + 4, w + 8, w + 12
 // share the lanes 32 (w % 4) ..; each takes 32 of the 128 columns: the element-wise work has no reduction
@@ -49,13 +51,13 @@ constexpr int kB1Stages = 3, kB2Stages = 2;
 
 // shared memory map (bytes from the 1024-aligned base)
 constexpr int kOffA1 = 0, kOffA2 = kBwdTileBytes, kOffB1 = 2 * kBwdTileBytes, kOffB2 = kOffB1 + kB1Stages * kBwdTileBytes;
-constexpr int kOffBars = kOffB2 + kB2Stages * kBwdTileBytes;                          // 16 barriers
-constexpr int kOffMisc = kOffBars + 128;                                              // TMEM slot, abort flags
+constexpr int kOffBars = kOffB2 + kB2Stages * kBwdTileBytes;                          // 18 barriers
+constexpr int kOffMisc = kOffBars + 192;                                              // TMEM slot, abort flags
 constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [2][lse, delta][128] per-query scalars
 constexpr int kBwdTcLayoutBytes = kOffRow + 2 * 2 * 128 * 4;
 constexpr int kBwdTcSmem = 232448;              // the whole opt-in window: the layout needs all but 832 bytes of it
 enum : int { BB_AFULL = 0, BB_B1FULL = 1, BB_B2FULL = 4, BB_XFULL = 6, BB_YFULL = 7, BB_PA = 8, BB_PB = 9, BB_OFULL = 10,
-             BB_B1EMPTY = 11, BB_B2EMPTY = 14 };
+             BB_B1EMPTY = 11, BB_B2EMPTY = 14, BB_YFULL2 = 16, BB_PB2 = 17 };
 static_assert(kBwdTcLayoutBytes <= kBwdTcSmem, "shared memory layout");
 
 // Optional event trace (compile with -DKSA_BWD_TRACE): one CTA of the dQ kernel records (event id, clock)
@@ -139,8 +141,10 @@ __device__ __forceinline__ void bt_init(const BtSmem& sm, int tid, int warp)
         for (int s = 0; s < kB2Stages; ++s) { mbar_init(sm.bar(BB_B2FULL + s), 1); mbar_init(sm.bar(BB_B2EMPTY + s), 1); }
         mbar_init(sm.bar(BB_XFULL), 1);
         mbar_init(sm.bar(BB_YFULL), 1);
+        mbar_init(sm.bar(BB_YFULL2), 1);
         mbar_init(sm.bar(BB_PA), 16);
         mbar_init(sm.bar(BB_PB), 16);
+        mbar_init(sm.bar(BB_PB2), 16);
         mbar_init(sm.bar(BB_OFULL), 1);
         bt_st_shared(sm.abort_addr(), 0u);
         bt_st_shared(sm.abort_addr() + 4, 0u);
@@ -251,15 +255,14 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     const int quarter = warp & 3, cg = warp >> 2;                        // row warps: lanes 32 quarter ..; columns 32 cg ..
     const bool scalar_writer = warp < 16 && quarter == 0;
     float n_lse = 0.f, n_dl = 0.f;                                        // the writer lane's values for the next tile
-    auto fetch = [&](int j) {
-        int qt, h;
-        pair_of(j, qt, h);
+    auto fetch = [&](int qt, int g) {                                     // pair (query tile qt, head g of the group)
+        const int h = hk * G + g;
         const size_t r = (size_t)h * a.text_rows + sq.text_off + (size_t)qt * 128 + 32 * cg + lane;
         n_lse = a.lse_t[r];                                               // +inf on padding rows: P = 0 there
         n_dl = a.delta_t[r];
     };
     if (scalar_writer) {                                                  // tile 0: visible to all after the first barrier
-        fetch(0);
+        fetch(seg0, 0);
         rows[32 * cg + lane] = n_lse;
         rows[128 + 32 * cg + lane] = n_dl;
     }
@@ -322,13 +325,18 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         const int kq = key / (summ ? a.m : a.k);                          // the key's chunk
         const int kq_first = (kt * 128) / (summ ? a.m : a.k), kq_last = (kt * 128 + 127) / (summ ? a.m : a.k);
         bool alive = true;
+        // The streamed tiles walk the pairs (query tile, head of the group) in order; the chunk of the block's first
+        // query, i0 = 128 qt + 32 cg, is kept as quotient and remainder by k and advanced by 128 per query tile
+        // (integer divisions are slow, and this loop is the warps' critical path).
+        const int step_q = 128 / a.k, step_r = 128 - step_q * a.k, q31 = 31 / a.k, r31 = 31 - q31 * a.k;
+        int qt = seg0, g = 0;
+        int iq0 = (seg0 * 128 + 32 * cg) / a.k, ir0 = (seg0 * 128 + 32 * cg) - iq0 * a.k;
         for (int j = 0; j < J && alive; ++j) {
-            int qt, h;
-            pair_of(j, qt, h);
-            if (scalar_writer && j + 1 < J) fetch(j + 1);                 // lands while this tile is worked on
+            if (scalar_writer && j + 1 < J) fetch(g + 1 == G ? qt + 1 : qt, g + 1 == G ? 0 : g + 1);   // lands while this tile is worked on
             const float* lse_c = rows + (j & 1) * 256 + 32 * cg;          // this warp's 32 columns
             const float* dl_c = lse_c + 128;
             const int i0 = qt * 128 + 32 * cg;                            // first query of the block
+            const int iq1 = iq0 + q31 + (ir0 + r31 >= a.k ? 1 : 0);       // chunk of the block's last query
             // ---------------- phase A: P^T = exp2(S^T scale - lse) ----------------
             if (!bt_wait_warp(sm.bar(BB_XFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
             tc_fence_after();
@@ -336,7 +344,6 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             if (warp == 0 && lane == 0 && j >= 1) mbar_arrive(sm.bar(BB_B2EMPTY + ((j - 1) & 1)));
             // all pairs of the block visible / none (rows past the streams drop out by themselves: zero K / V
             // rows are discarded at the end, padding queries have lse = +inf)
-            const int iq0 = i0 / a.k, ir0 = i0 - iq0 * a.k, iq1 = (i0 + 31) / a.k;
             bool full, none;
             if (!summ) {
                 full = kt * 128 + 127 <= i0 && iq1 - kq_first <= a.C;
@@ -424,6 +431,11 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     mbar_arrive(sm.bar(BB_PB));
                 }
             }
+            if (++g == G) {                                               // next query tile
+                g = 0; ++qt;
+                iq0 += step_q; ir0 += step_r;
+                if (ir0 >= a.k) { ir0 -= a.k; ++iq0; }
+            }
         }
         if (alive && bt_wait_warp(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull, lane)) {
             tc_fence_after();
@@ -485,7 +497,12 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
     if (!bt_layout(sm, bsm_raw, a.status)) return;
     bt_init(sm, tid, warp);
     const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
-    const uint32_t tX = tmem, tY = tmem + 128u, tDQ = tmem + 256u;
+    const uint32_t tX = tmem, tDQ = tmem + 256u;
+    auto tY = [&](int j) -> uint32_t { return tmem + ((j & 1) ? 384u : 128u); };   // dP of tile j, then dS in place
+    auto y_full = [&](int j) -> uint32_t { return sm.bar((j & 1) ? BB_YFULL2 : BB_YFULL); };
+    // likewise one phase B barrier per Y buffer: with both products of tile j + 1 issued early, a warp may finish
+    // tile j + 1 before another has finished tile j, and must not arrive in its phase
+    auto p_b = [&](int j) -> uint32_t { return sm.bar((j & 1) ? BB_PB2 : BB_PB); };
 
     if (warp == 16) {
         // =============================== TMA producer ===============================
@@ -519,20 +536,22 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             if (alive) alive = bt_wait(sm.bar(BB_B1FULL), 0, abort_addr, a.status, kStatusWaitQFull);
             if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
-            if (alive) { bt_product(tY, sm.a2(), sm.b2(0)); tc_commit(sm.bar(BB_YFULL)); }
+            if (alive) { bt_product(tY(0), sm.a2(), sm.b2(0)); tc_commit(y_full(0)); }
             for (int j = 0; j < J && alive; ++j) {
-                // later stages were checked by row warp 0 before its arrivals
+                // later stages were checked by row warp 0 before its arrival
                 if (j + 1 < J) {
-                    // phase A of tile j has read X into registers
+                    // phase A of tile j has read X into registers; the other Y buffer was read by dQ += dS K_{j-1}
                     if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                     tc_fence_after();
                     bt_product(tX, sm.a1(), sm.b1((j + 1) % kB1Stages));
                     tc_commit(sm.bar(BB_XFULL));
+                    bt_product(tY(j + 1), sm.a2(), sm.b2((j + 1) & 1));
+                    tc_commit(y_full(j + 1));
                 }
-                if (!bt_wait(sm.bar(BB_PB), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                if (!bt_wait(p_b(j), (j >> 1) & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                 tc_fence_after();
-                bt_accumulate(tDQ, tY, sm.b1(j % kB1Stages), j == 0);                       // dQ += dS K_j
-                if (j + 1 < J) { bt_product(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
+                bt_accumulate(tDQ, tY(j), sm.b1(j % kB1Stages), j == 0);                    // dQ += dS K_j
+                tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // K_j is free after that
             }
             tc_commit(sm.bar(BB_OFULL));
         }
@@ -540,7 +559,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         // =============================== query rows =================================
         const int quarter = warp & 3, cg = warp >> 2;                    // lanes 32 quarter ..; columns 32 cg ..
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-        const uint32_t tXc = tX + lane_sel + cg * 32, tYc = tY + lane_sel + cg * 32;    // this warp's 32 x 32 block
+        const uint32_t tXc = tX + lane_sel + cg * 32;                     // this warp's 32 x 32 block
         const int i_w0 = i_first + quarter * 32, i = i_w0 + lane;         // this thread's query row
         const size_t r = (size_t)h * a.text_rows + sq.text_off + i;
         const float lse2 = a.lse_t[r], dl = a.delta_t[r];                 // +inf / 0 on padding rows: P = 0 there
@@ -551,12 +570,24 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         uint32_t bt_n = 0;
 #endif
         bool alive = true;
+        // The chunk of the block's first key, kc0 = key0 + 32 cg, is kept as quotient and remainder by the keys per
+        // chunk of its stream and advanced by 128 per tile; divisions only where the stream starts (integer
+        // divisions are slow, and this loop is the warps' critical path).
+        int cdiv = 1, kq0 = 0, kr0 = 0, step_q = 0, step_r = 0, q31 = 0, r31 = 0;
         for (int j = 0; j < J; ++j) {
             bool is_summ; int key0;
             tile_of(j, is_summ, key0);
             const int kc0 = key0 + 32 * cg;                               // first key of this warp's block
-            const int cdiv = is_summ ? a.m : a.k;                         // keys per chunk in this stream
-            const int kq0 = kc0 / cdiv, kr0 = kc0 - kq0 * cdiv, kq1 = (kc0 + 31) / cdiv;
+            if (j == 0 || j == n_s) {                                     // first tile of the summary / the text stream
+                cdiv = is_summ ? a.m : a.k;                               // keys per chunk in this stream
+                kq0 = kc0 / cdiv; kr0 = kc0 - kq0 * cdiv;
+                step_q = 128 / cdiv; step_r = 128 - step_q * cdiv;
+                q31 = 31 / cdiv; r31 = 31 - q31 * cdiv;
+            } else {
+                kq0 += step_q; kr0 += step_r;
+                if (kr0 >= cdiv) { kr0 -= cdiv; ++kq0; }
+            }
+            const int kq1 = kq0 + q31 + (kr0 + r31 >= cdiv ? 1 : 0);      // chunk of the block's last key
             // the warp's 32 x 32 block: all visible, none, or mixed (zero rows past a stream add nothing to dQ).
             // Text key t is visible to row i iff t <= i and chunk(i) - chunk(t) <= C; summary key s iff
             // chunk(i) - chunk(s) > C (Eq. 3)
@@ -581,8 +612,10 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {                                              // X may be overwritten from here on
-                if (warp == 0 && j + 1 < J)                                // warp 0 vouches for the stage of X_{j+1}
+                if (warp == 0 && j + 1 < J) {                              // warp 0 vouches for the stages of X_{j+1} and Y_{j+1}
                     bt_wait(sm.bar(BB_B1FULL + (j + 1) % kB1Stages), ((j + 1) / kB1Stages) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
+                    bt_wait(sm.bar(BB_B2FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
+                }
                 mbar_arrive(sm.bar(BB_PA));
             }
             KSA_BT(bt_role, 11);
@@ -607,14 +640,12 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             }
             KSA_BT(bt_role, 12);
             // ---------------- phase B: dS = P (dP - delta) ----------------
-            if (!bt_wait_warp(sm.bar(BB_YFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
+            // one barrier per Y buffer: Y_{j+1} may be complete before a warp gets here for Y_j
+            if (!bt_wait_warp(y_full(j), (j >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
             KSA_BT(bt_role, 13);
             tc_fence_after();
-            // Y_j is complete: its V stage is free, and so is the K stage of tile j - 1 (dQ += dS K_{j-1} came before it)
-            if (warp == 0 && lane == 0) {
-                mbar_arrive(sm.bar(BB_B2EMPTY + (j & 1)));
-                if (j >= 1) mbar_arrive(sm.bar(BB_B1EMPTY + (j - 1) % kB1Stages));
-            }
+            if (warp == 0 && lane == 0) mbar_arrive(sm.bar(BB_B2EMPTY + (j & 1)));          // Y_j is complete: its V stage is free
+            const uint32_t tYc = tY(j) + lane_sel + cg * 32;
             uint32_t dd[16];
             if (none) {
 #pragma unroll
@@ -636,11 +667,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                if (warp == 0 && j + 1 < J)                                // warp 0 vouches for the stage of Y_{j+1}
-                    bt_wait(sm.bar(BB_B2FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
-                mbar_arrive(sm.bar(BB_PB));
-            }
+            if (lane == 0) mbar_arrive(p_b(j));
             KSA_BT(bt_role, 14);
         }
 #ifdef KSA_BWD_TRACE
