@@ -457,7 +457,7 @@ def run_backward(args):
         "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
         "roofline": {"bound": "tensor", "achieved": val, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                      "frac": val / peaks["bf16_sustained"], "traffic": None,
-                     "peak_source": f"of {peaks['source']} (sustained bf16 GEMM)", "kernel": "ksa_bwd_dq_kernel + ksa_bwd_dkv_kernel (mma.sync; whole step)"},
+                     "peak_source": f"of {peaks['source']} (sustained bf16 GEMM)", "kernel": "ksa_bwd_dq_tc_kernel + ksa_bwd_dkv_tc_kernel (tcgen05; whole step incl. pack, prep, summary rows, finish)"},
         "e2e": None, "cpu_baseline": None,
     }
     print(json.dumps(line))

@@ -237,7 +237,8 @@ int ksa_schedule_dump(ksa_ctx* ctx, const ksa_params* p, ksa_tile_rec* recs, int
 
 /* ---- diagnostics -------------------------------------------------------------------- */
 /* Reads (with a blocking copy) the device status word written by bounded waits:
- * 0 = no wait ever gave up; otherwise a code naming the first wait that did. */
+ * 0 = no wait ever gave up; otherwise a code naming the first wait that did (9: a kernel found
+ * that its shared-memory layout does not fit the window it was given, and did nothing). */
 int ksa_last_device_status(ksa_ctx* ctx, int32_t* status);
 /* Clears the device status word (blocking copy). */
 int ksa_clear_device_status(ksa_ctx* ctx);

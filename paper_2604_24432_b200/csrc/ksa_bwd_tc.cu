@@ -60,8 +60,9 @@ enum : int { BB_AFULL = 0, BB_B1FULL = 1, BB_B2FULL = 4, BB_XFULL = 6, BB_YFULL 
              BB_B1EMPTY = 11, BB_B2EMPTY = 14, BB_YFULL2 = 16, BB_PB2 = 17 };
 static_assert(kBwdTcLayoutBytes <= kBwdTcSmem, "shared memory layout");
 
-// Optional event trace (compile with -DKSA_BWD_TRACE): one CTA of the dQ kernel records (event id, clock)
-// pairs for lane 0 of every row warp; ksa_debug_read_bwd_trace() copies them out.
+// Optional event trace (compile with -DKSA_BWD_TRACE=1 for the dQ kernel, =3 for the dK / dV kernel over summary
+// keys): one CTA records (event id, clock) pairs for lane 0 of every row warp; ksa_debug_read_bwd_trace() copies
+// them out.
 #ifdef KSA_BWD_TRACE
 constexpr int kBtEvents = 4096;
 __device__ uint2 g_btrace[17][kBtEvents];         // role 0: MMA issuer (sums only); 1 + w: row warp w
@@ -329,6 +330,11 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         // query, i0 = 128 qt + 32 cg, is kept as quotient and remainder by k and advanced by 128 per query tile
         // (integer divisions are slow, and this loop is the warps' critical path).
         const int step_q = 128 / a.k, step_r = 128 - step_q * a.k, q31 = 31 / a.k, r31 = 31 - q31 * a.k;
+#ifdef KSA_BWD_TRACE
+        const bool bt_on = KSA_BWD_TRACE == 3 && summ && blockIdx.x == 1 && blockIdx.y == 4 && blockIdx.z == 0 && lane == 0;
+        const int bt_role = 1 + warp;
+        uint32_t bt_n = 0;
+#endif
         int qt = seg0, g = 0;
         int iq0 = (seg0 * 128 + 32 * cg) / a.k, ir0 = (seg0 * 128 + 32 * cg) - iq0 * a.k;
         for (int j = 0; j < J && alive; ++j) {
@@ -339,6 +345,7 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             const int iq1 = iq0 + q31 + (ir0 + r31 >= a.k ? 1 : 0);       // chunk of the block's last query
             // ---------------- phase A: P^T = exp2(S^T scale - lse) ----------------
             if (!bt_wait_warp(sm.bar(BB_XFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
+            KSA_BT(bt_role, 10);
             tc_fence_after();
             // X_j was issued after dV += P^T dO_{j-1}: that tile's dO stage is free
             if (warp == 0 && lane == 0 && j >= 1) mbar_arrive(sm.bar(BB_B2EMPTY + ((j - 1) & 1)));
@@ -352,38 +359,40 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                 full = iq0 - kq_last > a.C;
                 none = iq1 - kq_first <= a.C;
             }
-            float p[32];
+            uint32_t x0[16], x1[16];                                      // S^T, then P^T in place (fp32 bits), kept for phase B
             if (none) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) p[c] = 0.f;
+                for (int c = 0; c < 16; ++c) x0[c] = x1[c] = 0u;
             } else {
+                tmem_ld16(tXc, x0);
+                tmem_ld16(tXc + 16, x1);
+                tc_wait_ld();
+                KSA_BT(bt_role, 11);
+                if (full) {
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t xs[16];
-                    tmem_ld16(tXc + half * 16, xs);
-                    tc_wait_ld();
-                    if (full) {
+                    for (int c = 0; c < 16; ++c) {
+                        x0[c] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(x0[c]), a.scale_log2, -lse_c[c])));
+                        x1[c] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(x1[c]), a.scale_log2, -lse_c[16 + c])));
+                    }
+                } else {
+                    int iq = iq0, ir = ir0;                               // chunk of query i0 + c, counted up from i0's
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            p[half * 16 + c] = ex2_approx(fmaf(__uint_as_float(xs[c]), a.scale_log2, -lse_c[half * 16 + c]));
-                    } else {
-                        // chunk of query i0 + c, found by counting up from i0's
-                        int iq = iq0, ir = ir0 + half * 16;
-                        while (ir >= a.k) { ir -= a.k; ++iq; }
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const bool vis = summ ? (iq - kq > a.C) : (key <= i0 + half * 16 + c && iq - kq <= a.C);
-                            const float t = fmaf(__uint_as_float(xs[c]), a.scale_log2, -lse_c[half * 16 + c]);
-                            p[half * 16 + c] = ex2_approx(vis ? t : -INFINITY);
-                            if (++ir == a.k) { ir = 0; ++iq; }
-                        }
+                    for (int c = 0; c < 32; ++c) {
+                        uint32_t& xc = c < 16 ? x0[c & 15] : x1[c & 15];
+                        const bool vis = summ ? (iq - kq > a.C) : (key <= i0 + c && iq - kq <= a.C);
+                        const float t = fmaf(__uint_as_float(xc), a.scale_log2, -lse_c[c]);
+                        xc = __float_as_uint(ex2_approx(vis ? t : -INFINITY));
+                        if (++ir == a.k) { ir = 0; ++iq; }
                     }
                 }
             }
             {
                 uint32_t pp[16];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) pp[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+                for (int c = 0; c < 8; ++c) {
+                    pp[c] = pack_bf16x2(__uint_as_float(x0[2 * c]), __uint_as_float(x0[2 * c + 1]));
+                    pp[8 + c] = pack_bf16x2(__uint_as_float(x1[2 * c]), __uint_as_float(x1[2 * c + 1]));
+                }
                 tmem_st16(tXc, pp);                                       // over the block's own first 16 columns
                 // X_j was complete, so every warp is past phase A of tile j - 1: its lse buffer may be overwritten
                 // (the arrival below publishes the values: X_{j+1} is only issued after it)
@@ -397,8 +406,10 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     mbar_arrive(sm.bar(BB_PA));
                 }
             }
+            KSA_BT(bt_role, 12);
             // ---------------- phase B: dS^T = P^T (dP^T - delta) ----------------
             if (!bt_wait_warp(sm.bar(BB_YFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
+            KSA_BT(bt_role, 13);
             tc_fence_after();
             // Y_j was issued after dK += dS^T Q_{j-1}: that tile's Q stage is free
             if (warp == 0 && lane == 0 && j >= 1) mbar_arrive(sm.bar(BB_B1EMPTY + (j - 1) % kB1Stages));
@@ -414,9 +425,11 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                         tmem_ld16(tYc + half * 16, ys);
                         tc_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 16; c += 2)
-                            dd[half * 8 + (c >> 1)] = pack_bf16x2(p[half * 16 + c] * (__uint_as_float(ys[c]) - dl_c[half * 16 + c]),
-                                                                  p[half * 16 + c + 1] * (__uint_as_float(ys[c + 1]) - dl_c[half * 16 + c + 1]));
+                        for (int c = 0; c < 16; c += 2) {
+                            const float p0 = __uint_as_float(half ? x1[c] : x0[c]), p1 = __uint_as_float(half ? x1[c + 1] : x0[c + 1]);
+                            dd[half * 8 + (c >> 1)] = pack_bf16x2(p0 * (__uint_as_float(ys[c]) - dl_c[half * 16 + c]),
+                                                                  p1 * (__uint_as_float(ys[c + 1]) - dl_c[half * 16 + c + 1]));
+                        }
                     }
                 }
                 tmem_st16(tYc, dd);
@@ -431,12 +444,16 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     mbar_arrive(sm.bar(BB_PB));
                 }
             }
+            KSA_BT(bt_role, 14);
             if (++g == G) {                                               // next query tile
                 g = 0; ++qt;
                 iq0 += step_q; ir0 += step_r;
                 if (ir0 >= a.k) { ir0 -= a.k; ++iq0; }
             }
         }
+#ifdef KSA_BWD_TRACE
+        if (bt_on) g_btrace_cnt[bt_role] = bt_n;
+#endif
         if (alive && bt_wait_warp(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull, lane)) {
             tc_fence_after();
             // odd cg: scale * dK, even cg: dV; cg / 2 picks the 64-element half of the row
@@ -565,7 +582,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         const float lse2 = a.lse_t[r], dl = a.delta_t[r];                 // +inf / 0 on padding rows: P = 0 there
         const int iq = i / a.k, iq_w0 = i_w0 / a.k, iq_w1 = (i_w0 + 31) / a.k;
 #ifdef KSA_BWD_TRACE
-        const bool bt_on = blockIdx.x == 8 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0;
+        const bool bt_on = KSA_BWD_TRACE == 1 && blockIdx.x == 8 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0;
         const int bt_role = 1 + warp;
         uint32_t bt_n = 0;
 #endif
