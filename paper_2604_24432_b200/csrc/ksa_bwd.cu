@@ -378,27 +378,38 @@ __global__ void __launch_bounds__(128) ksa_bwd_dkv_kernel(BwdArgs a, int summ)
 // =================================================================================================
 __global__ void __launch_bounds__(256) ksa_bwd_prep_kernel(BwdArgs a)
 {
+    // One 16-byte vector (8 elements) per lane: D / 8 lanes make up a (row, head) unit, a warp holds 32 / (D / 8)
+    // units (consecutive heads of one row first: those are contiguous in dout / out).
     const SeqInfo sq = a.seqs[blockIdx.y];
     const int lane = threadIdx.x & 31;
+    const int lanes_per_unit = a.D / 8, units_per_warp = 32 / lanes_per_unit;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (warp >= (int64_t)sq.text_pad * a.Hq) return;
-    const int i = (int)(warp / a.Hq), h = (int)(warp % a.Hq);
+    const int64_t unit = warp * units_per_warp + lane / lanes_per_unit;
+    const int sub = lane % lanes_per_unit;
+    const bool live = unit < (int64_t)sq.text_pad * a.Hq;
+    const int i = live ? (int)(unit / a.Hq) : 0, h = live ? (int)(unit % a.Hq) : 0;
     const size_t prow = (size_t)h * a.text_rows + sq.text_off + i;
-    const int E = a.D / 32;                      // 2 or 4 elements per lane
-    uint16_t* dst = a.dot + prow * a.D + lane * E;
-    if (i >= sq.n_text) {
-        for (int e = 0; e < E; ++e) dst[e] = 0;
-        if (lane == 0) { a.lse_t[prow] = INFINITY; a.delta_t[prow] = 0.f; }
-        return;
-    }
-    const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * (a.k + a.m) + (i % a.k);
-    const uint16_t* g = a.dout + aug * a.do_st + (int64_t)h * a.do_sh + lane * E;
-    const uint16_t* o = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
     float d = 0.f;
-    for (int e = 0; e < E; ++e) { dst[e] = g[e]; d = fmaf(b_bf2f(g[e]), b_bf2f(o[e]), d); }
+    float lse2 = INFINITY;
+    uint4 gv = make_uint4(0u, 0u, 0u, 0u);
+    const bool real = live && i < sq.n_text;
+    if (real) {
+        const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * (a.k + a.m) + (i % a.k);
+        gv = *reinterpret_cast<const uint4*>(a.dout + aug * a.do_st + (int64_t)h * a.do_sh + sub * 8);
+        const uint4 ov = *reinterpret_cast<const uint4*>(a.out + aug * a.o_st + (int64_t)h * a.o_sh + sub * 8);
+        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, ow[4] = {ov.x, ov.y, ov.z, ov.w};
 #pragma unroll
-    for (int s = 16; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
-    if (lane == 0) { a.lse_t[prow] = a.lse[(int64_t)h * a.total_aug + aug] * 1.4426950408889634f; a.delta_t[prow] = d; }
+        for (int e = 0; e < 4; ++e) {
+            d = fmaf(__uint_as_float(gw[e] << 16), __uint_as_float(ow[e] << 16), d);
+            d = fmaf(__uint_as_float(gw[e] & 0xffff0000u), __uint_as_float(ow[e] & 0xffff0000u), d);
+        }
+        if (sub == 0) lse2 = a.lse[(int64_t)h * a.total_aug + aug] * 1.4426950408889634f;
+    }
+    // sum over the lanes of the unit (whole warps take part: no early exit above)
+    for (int s = lanes_per_unit >> 1; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
+    if (!live) return;
+    *reinterpret_cast<uint4*>(a.dot + prow * a.D + sub * 8) = gv;        // zeros on padding rows
+    if (sub == 0) { a.lse_t[prow] = lse2; a.delta_t[prow] = real ? d : 0.f; }
 }
 
 // =================================================================================================
@@ -506,7 +517,8 @@ cudaError_t setup_bwd()
 
 cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream)
 {
-    const int64_t warps = (int64_t)a.max_text_pad * a.Hq;
+    const int64_t units = (int64_t)a.max_text_pad * a.Hq;                // (row, head) units, 32 / (D / 8) per warp
+    const int64_t warps = (units * (a.D / 8) + 31) / 32;
     dim3 grid((unsigned)((warps + 7) / 8), (unsigned)a.num_seqs, 1);
     ksa_bwd_prep_kernel<<<grid, 256, 0, stream>>>(a);
     return cudaGetLastError();
