@@ -67,3 +67,52 @@ def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     _check("dq", dq.double().cpu().numpy(), rdq)
     _check("dk", dk.double().cpu().numpy(), rdk)
     _check("dv", dv.double().cpu().numpy(), rdv)
+
+
+@pytest.mark.parametrize("workload", ["32k", "128k"])
+def test_backward_full_size_identities(ctx, workload):
+    """Full-size workloads, in the launch configuration the bench times: two identities that hold for the exact
+    gradients at any size and involve every element of dq, dk and dv.
+
+    (a) The scores only see q k^T, so scaling q by t and k by 1/t changes nothing: d/dt at t = 1 gives
+        sum <q, dq> = sum <k, dk> over the rows and the query heads of every KV head.
+    (b) out is linear in v: sum <v, dv> = sum <out, dout> over the rows and the query heads of every KV head.
+    Both sides are sums of terms of either sign; bf16 gradients (relative error about 2^-9 per element, random
+    sign) keep the difference far below 2e-3 of the sum of the absolute terms."""
+    wl = synth.WORKLOADS[workload]
+    lay = synth.LAYOUT_P
+    dev = torch.device("cuda", 0)
+    prob = ksa.Problem(wl.text_lens, lay.k, lay.m, lay.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total = ksa.total_aug_len(prob)
+    q, kk, v = synth.make_qkv(wl, total)
+    qd, kd, vd = q.to(dev), kk.to(dev), v.to(dev)
+    g = torch.Generator("cpu").manual_seed(5)
+    gd = torch.randn((total, wl.Hq, wl.D), generator=g, dtype=torch.float32).to(torch.bfloat16).to(dev)
+    out = torch.empty_like(qd); lse = torch.empty((wl.Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx.clear_device_status()
+    ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws)
+    dq = torch.full_like(qd, 7.0); dk = torch.full_like(kd, 7.0); dv = torch.full_like(vd, 7.0)
+    wsb = torch.full((ksa.bwd_workspace_bytes(prob),), 0xFF, dtype=torch.uint8, device=dev)
+    ctx.attn_bwd(prob, qd, kd, vd, out, lse, gd, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for t in (dq, dk, dv):
+        assert torch.isfinite(t.float()).all()
+    G = wl.Hq // wl.Hkv
+
+    def per_kv_head(a, b, heads_per_kv):       # sum over rows and elements of a * b, and of |a * b|, per KV head
+        prod = (a.double() * b.double()).sum(dim=2)                        # [rows, heads]
+        absum = (a.double() * b.double()).abs().sum(dim=2)
+        prod = prod.sum(dim=0).reshape(wl.Hkv, heads_per_kv).sum(dim=1)
+        absum = absum.sum(dim=0).reshape(wl.Hkv, heads_per_kv).sum(dim=1)
+        return prod.cpu().numpy(), absum.cpu().numpy()
+
+    qdq, qabs = per_kv_head(qd, dq, G)
+    kdk, kabs = per_kv_head(kd, dk, 1)
+    vdv, vabs = per_kv_head(vd, dv, 1)
+    odo, oabs = per_kv_head(out, gd, G)
+    assert (np.abs(qdq - kdk) <= 2e-3 * (qabs + kabs)).all(), (qdq, kdk, qabs)
+    assert (np.abs(vdv - odo) <= 2e-3 * (vabs + oabs)).all(), (vdv, odo, vabs)
+    # the identities are not met by zeros only: the gradients have their expected size
+    assert (qabs > 0).all() and (vabs > 0).all()
