@@ -42,6 +42,8 @@ def _check(name, got, ref):
     ([2100, 640], 8, 1, 16, 8, 2, 128, 0),            # several query segments per summary key tile
     ([2500], 64, 8, 4, 4, 2, 128, 0),                 # long chunks with 8 summaries each
     ([600, 9], 8, 1, 0, 4, 2, 128, 0),                # no window beyond the own chunk
+    ([900], 8, 1, 1000, 4, 2, 128, 0),                # window longer than the sequence: plain causal attention
+    ([5, 130, 64, 1, 257], 8, 1, 4, 8, 1, 128, 0),    # many short sequences, one KV head for 8 query heads
 ])
 def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
