@@ -110,7 +110,7 @@ def dist_env():
 
 def workload_and_layout(args):
     wl = synth.WORKLOADS[args.workload]
-    layout = synth.LAYOUT_P if args.layout == "P" else synth.LAYOUT_G
+    layout = {"P": synth.LAYOUT_P, "G": synth.LAYOUT_G, "F": synth.LAYOUT_F}[args.layout]
     return wl, layout
 
 
@@ -480,7 +480,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="128k", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--layout", default="P", choices=["P", "G"])
+    ap.add_argument("--layout", default="P", choices=["P", "G", "F"],
+                    help="P, G: the paper's KSA layouts; F: full causal attention (the hybrid stack's full layers)")
     ap.add_argument("--oracle-rows", type=int, default=3000)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")

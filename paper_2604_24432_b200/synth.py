@@ -31,6 +31,9 @@ class Layout:
 LAYOUT_P = Layout("P", 8, 1, 128)
 # Same 8x compression and 1,024-token window with 64-token chunks and 8 summaries each.
 LAYOUT_G = Layout("G", 64, 8, 16)
+# The full-attention layers of the hybrid stack (one in four, Table 2): no summary tokens, a window that covers
+# every chunk, i.e. plain causal attention through the same entry points.
+LAYOUT_F = Layout("F", 8, 0, 1 << 20)
 
 
 @dataclass(frozen=True)
