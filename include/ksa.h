@@ -162,6 +162,10 @@ int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* byt
  *   dk, dv              DEVICE bf16, layouts and strides of k and v; every row is written
  *   workspace           DEVICE, >= ksa_bwd_workspace_bytes, 256-byte aligned, scratch
  * Asynchronous on cuda_stream.  KSA_FLAG_REFERENCE_KERNEL is not accepted here.
+ * With head_dim 128 and every sequence a whole number of chunks (the no-pack case of
+ * ksa_attn_fwd) the tensor-core kernels read q, k, v and dout in place: rows of other
+ * sequences that share a 128-row tile are masked, so all of these tensors must hold finite
+ * values everywhere.
  * Errors as for ksa_attn_fwd.
  */
 int ksa_attn_bwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, const void* out, const float* lse,

@@ -722,9 +722,11 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
         if ((e = setup_bwd()) != cudaSuccess) return cuda_fail(ctx, e);
         bwd_ready = true;
     }
-    // packed streams of the forward pass (text Q, K, V and summary K, V)
+    // packed streams of the forward pass (text Q, K, V and summary K, V) -- not needed when the tensor-core kernels
+    // can read whole tiles straight from the caller's tensors (the no-pack case of the forward pass)
+    const bool direct = p->head_dim == 128 && direct_ok(p);
     KernelArgs fa = make_args(ctx, p, q, k, v, dq /* unused */, const_cast<float*>(lse), workspace, bl.fwd);
-    if ((e = launch_pack(fa, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if (!direct && (e = launch_pack(fa, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     BwdArgs a{};
     a.seqs = ctx->d_seqs; a.num_seqs = p->num_seqs;
     a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.C = p->window_chunks;
@@ -743,6 +745,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     a.dot = (uint16_t*)(ws + bl.dot); a.lse_t = (float*)(ws + bl.lse_t); a.delta_t = (float*)(ws + bl.delta_t);
     a.dkt = (float*)(ws + bl.dkt); a.dvt = (float*)(ws + bl.dvt); a.dks = (float*)(ws + bl.dks); a.dvs = (float*)(ws + bl.dvs);
     a.status = ctx->d_status;
+    a.direct = direct ? 1 : 0;
     // the four accumulators are contiguous in the workspace: one clear
     if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
@@ -755,12 +758,28 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
             bwd_tc_ready = true;
         }
         BwdMaps bm;
-        struct { CUtensorMap* map; const void* base; int64_t rows; int H; } streams[6] = {
-            {&bm.qt, a.qt, a.text_rows, a.Hq},   {&bm.dot, a.dot, a.text_rows, a.Hq},
-            {&bm.kt, a.kt, a.text_rows, a.Hkv},  {&bm.vt, a.vt, a.text_rows, a.Hkv},
-            {&bm.ks, a.ks, a.summ_rows, a.Hkv},  {&bm.vs, a.vs, a.summ_rows, a.Hkv}};
-        for (auto& t : streams)
-            if ((rc = encode_stream_map(ctx, t.map, const_cast<void*>(t.base), a.D, t.rows, t.H)) != KSA_OK) return rc;
+        if (direct) {
+            // chunked views [D, rows per chunk, chunk, head] of the caller's tensors; summary rows start k rows into a chunk
+            const int s_len = a.k + a.m;
+            const int64_t chunks = a.total_aug / s_len;
+            if ((rc = encode_chunk_map(ctx, &bm.qt, a.q, a.D, a.k, s_len, chunks, a.Hq, a.q_st, a.q_sh)) != KSA_OK) return rc;
+            if ((rc = encode_chunk_map(ctx, &bm.dot, a.dout, a.D, a.k, s_len, chunks, a.Hq, a.do_st, a.do_sh)) != KSA_OK) return rc;
+            if ((rc = encode_chunk_map(ctx, &bm.kt, a.kx, a.D, a.k, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
+            if ((rc = encode_chunk_map(ctx, &bm.vt, a.v, a.D, a.k, s_len, chunks, a.Hkv, a.v_st, a.v_sh)) != KSA_OK) return rc;
+            if (a.m > 0) {
+                if ((rc = encode_chunk_map(ctx, &bm.ks, a.kx + (int64_t)a.k * a.k_st, a.D, a.m, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
+                if ((rc = encode_chunk_map(ctx, &bm.vs, a.v + (int64_t)a.k * a.v_st, a.D, a.m, s_len, chunks, a.Hkv, a.v_st, a.v_sh)) != KSA_OK) return rc;
+            } else {
+                bm.ks = bm.kt; bm.vs = bm.vt;    // never used: no summary tiles
+            }
+        } else {
+            struct { CUtensorMap* map; const void* base; int64_t rows; int H; } streams[6] = {
+                {&bm.qt, a.qt, a.text_rows, a.Hq},   {&bm.dot, a.dot, a.text_rows, a.Hq},
+                {&bm.kt, a.kt, a.text_rows, a.Hkv},  {&bm.vt, a.vt, a.text_rows, a.Hkv},
+                {&bm.ks, a.ks, a.summ_rows, a.Hkv},  {&bm.vs, a.vs, a.summ_rows, a.Hkv}};
+            for (auto& t : streams)
+                if ((rc = encode_stream_map(ctx, t.map, const_cast<void*>(t.base), a.D, t.rows, t.H)) != KSA_OK) return rc;
+        }
         if ((e = launch_bwd_dq_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         if ((e = launch_bwd_dkv_tc(a, bm, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     } else {
@@ -768,7 +787,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
         if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     }
     if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 5 + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
+    ctx->launches += (direct ? 4 : 5) + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
     return KSA_OK;
 }
 

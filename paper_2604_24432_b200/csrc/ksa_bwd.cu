@@ -374,7 +374,7 @@ __global__ void __launch_bounds__(128) ksa_bwd_dkv_kernel(BwdArgs a, int summ)
 }
 
 // =================================================================================================
-// preparation: text rows of dO into the packed layout, lse in log2 units, delta = <dO, O>
+// preparation: text rows of dO into the packed layout (not in direct mode), lse in log2 units, delta = <dO, O>
 // =================================================================================================
 __global__ void __launch_bounds__(256) ksa_bwd_prep_kernel(BwdArgs a)
 {
@@ -408,7 +408,7 @@ __global__ void __launch_bounds__(256) ksa_bwd_prep_kernel(BwdArgs a)
     // sum over the lanes of the unit (whole warps take part: no early exit above)
     for (int s = lanes_per_unit >> 1; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
     if (!live) return;
-    *reinterpret_cast<uint4*>(a.dot + prow * a.D + sub * 8) = gv;        // zeros on padding rows
+    if (!a.direct) *reinterpret_cast<uint4*>(a.dot + prow * a.D + sub * 8) = gv;        // zeros on padding rows
     if (sub == 0) { a.lse_t[prow] = lse2; a.delta_t[prow] = real ? d : 0.f; }
 }
 

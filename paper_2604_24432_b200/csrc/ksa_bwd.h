@@ -27,10 +27,12 @@ struct BwdArgs {
     float* dkt; float* dvt;     // [Hkv][text_rows][D] fp32
     float* dks; float* dvs;     // [Hkv][summ_rows][D] fp32
     int32_t* status;            // device status word of the context (bounded waits report here)
+    int32_t direct;             // tensor-core kernels read q, k, v, dout through chunked views: no packed copies
 };
 
-// Tensor maps of the packed streams for the tensor-core kernels (128-byte swizzle, boxes of 64 elements x
-// 128 rows): Q and dO per query head, K and V of both streams per KV head.
+// Tensor maps for the tensor-core kernels (128-byte swizzle, boxes of 64 elements x 128 rows): Q and dO per query
+// head, K and V of the text and the summary rows per KV head -- of the packed streams, or (direct mode) chunked
+// 4-D views of the caller's interleaved tensors.
 struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs; };
 
 // Packs the text rows of dO, lse (in log2 units) and delta = <dO, O>.

@@ -182,11 +182,23 @@ __device__ __forceinline__ void bt_accumulate(uint32_t tmem_d, uint32_t tmem_a, 
 }
 
 // ---- producer helpers (one thread) ----------------------------------------------------------------
-__device__ __forceinline__ void bt_load_tile(uint32_t dst, uint32_t bar, const CUtensorMap* map, int row, int head)
+// The two 64-column halves of a 128-row tile.  Packed streams: rows pos .. pos + 127 of a 3-D map.  Direct mode
+// (no packed copies: every sequence a whole number of chunks): chunks pos .. of a 4-D view [D, rows per chunk,
+// chunk, head] of the caller's interleaved tensor, whose box lands in shared memory as the same dense tile.
+__device__ __forceinline__ void bt_issue_tile(uint32_t dst, uint32_t bar, const CUtensorMap* map, int pos, int head, bool direct)
+{
+    if (direct) {
+        tma_load_4d(dst, map, bar, 0, 0, pos, head);
+        tma_load_4d(dst + 16384, map, bar, 64, 0, pos, head);
+    } else {
+        tma_load_3d(dst, map, bar, 0, pos, head);
+        tma_load_3d(dst + 16384, map, bar, 64, pos, head);
+    }
+}
+__device__ __forceinline__ void bt_load_tile(uint32_t dst, uint32_t bar, const CUtensorMap* map, int pos, int head, bool direct)
 {
     mbar_arrive_expect_tx(bar, (uint32_t)kBwdTileBytes);
-    tma_load_3d(dst, map, bar, 0, row, head);
-    tma_load_3d(dst + 16384, map, bar, 64, row, head);
+    bt_issue_tile(dst, bar, map, pos, head, direct);
 }
 // After an abort: leave no copy in flight.  Bounded waits (the second flag is never set) for the last fill of
 // every stage; filled1 / filled2 = B1 / B2 tiles whose load was issued.
@@ -275,22 +287,25 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         // =============================== TMA producer ===============================
         if (lane == 0) {
             prefetch_tensormap(&maps.qt); prefetch_tensormap(&maps.dot);
+            const bool direct = a.direct != 0;
+            const int q_step = direct ? 128 / a.k : 128, q_base = direct ? sq.chunk0 : sq.text_off;   // position of a query tile
             mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * kBwdTileBytes);
-            for (int h2 = 0; h2 < 2; ++h2) {
-                tma_load_3d(sm.a1() + h2 * 16384, summ ? &maps.ks : &maps.kt, sm.bar(BB_AFULL), h2 * 64, krow0, hk);
-                tma_load_3d(sm.a2() + h2 * 16384, summ ? &maps.vs : &maps.vt, sm.bar(BB_AFULL), h2 * 64, krow0, hk);
+            {
+                const int kpos = direct ? sq.chunk0 + kt * (128 / (summ ? a.m : a.k)) : krow0;
+                bt_issue_tile(sm.a1(), sm.bar(BB_AFULL), summ ? &maps.ks : &maps.kt, kpos, hk, direct);
+                bt_issue_tile(sm.a2(), sm.bar(BB_AFULL), summ ? &maps.vs : &maps.vt, kpos, hk, direct);
             }
             int filled1 = 0, filled2 = 0;
             bool ok = true;
             for (int j = 0; j < J && ok; ++j) {
                 int qt, h;
                 pair_of(j, qt, h);
-                const int row = sq.text_off + qt * 128;
+                const int pos = q_base + qt * q_step;
                 if (!(ok = bt_stage_free(sm, BB_B1EMPTY, kB1Stages, j, a.status))) break;
-                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), &maps.qt, row, h);
+                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), &maps.qt, pos, h, direct);
                 ++filled1;
                 if (!(ok = bt_stage_free(sm, BB_B2EMPTY, kB2Stages, j, a.status))) break;
-                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), &maps.dot, row, h);
+                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), &maps.dot, pos, h, direct);
                 ++filled2;
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, filled1, filled2, a.status);
@@ -525,22 +540,26 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         // =============================== TMA producer ===============================
         if (lane == 0) {
             prefetch_tensormap(&maps.kt); prefetch_tensormap(&maps.vt);
+            const bool direct = a.direct != 0;
             mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * kBwdTileBytes);
-            for (int h2 = 0; h2 < 2; ++h2) {
-                tma_load_3d(sm.a1() + h2 * 16384, &maps.qt, sm.bar(BB_AFULL), h2 * 64, sq.text_off + qt * 128, h);
-                tma_load_3d(sm.a2() + h2 * 16384, &maps.dot, sm.bar(BB_AFULL), h2 * 64, sq.text_off + qt * 128, h);
+            {
+                const int qpos = direct ? sq.chunk0 + qt * (128 / a.k) : sq.text_off + qt * 128;
+                bt_issue_tile(sm.a1(), sm.bar(BB_AFULL), &maps.qt, qpos, h, direct);
+                bt_issue_tile(sm.a2(), sm.bar(BB_AFULL), &maps.dot, qpos, h, direct);
             }
             int filled1 = 0, filled2 = 0;
             bool ok = true;
             for (int j = 0; j < J && ok; ++j) {
                 bool is_summ; int key0;
                 tile_of(j, is_summ, key0);
-                const int row = (is_summ ? sq.summ_off : sq.text_off) + key0;
+                // key0 / 128 tiles into its stream: rows of the packed stream, or chunks of the caller's tensor
+                const int pos = direct ? sq.chunk0 + (key0 >> 7) * (128 / (is_summ ? a.m : a.k))
+                                       : (is_summ ? sq.summ_off : sq.text_off) + key0;
                 if (!(ok = bt_stage_free(sm, BB_B1EMPTY, kB1Stages, j, a.status))) break;
-                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), is_summ ? &maps.ks : &maps.kt, row, hk);
+                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), is_summ ? &maps.ks : &maps.kt, pos, hk, direct);
                 ++filled1;
                 if (!(ok = bt_stage_free(sm, BB_B2EMPTY, kB2Stages, j, a.status))) break;
-                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), is_summ ? &maps.vs : &maps.vt, row, hk);
+                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), is_summ ? &maps.vs : &maps.vt, pos, hk, direct);
                 ++filled2;
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, filled1, filled2, a.status);

@@ -44,6 +44,11 @@ def _check(name, got, ref):
     ([600, 9], 8, 1, 0, 4, 2, 128, 0),                # no window beyond the own chunk
     ([900], 8, 1, 1000, 4, 2, 128, 0),                # window longer than the sequence: plain causal attention
     ([5, 130, 64, 1, 257], 8, 1, 4, 8, 1, 128, 0),    # many short sequences, one KV head for 8 query heads
+    # whole chunks everywhere: the tensor-core kernels read q, k, v, dout in place (no packed copies)
+    ([1024, 264, 8], 8, 1, 4, 4, 2, 128, 0),          # sequences that end inside a 128-row tile
+    ([1280], 64, 8, 4, 4, 2, 128, 0),
+    ([704, 48], 16, 0, 7, 4, 4, 128, 0),
+    ([640], 8, 1, 3, 4, 1, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
 ])
 def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
