@@ -57,6 +57,9 @@ __device__ unsigned long long g_cta_span[2][256];   // start / end of every CTA 
 constexpr int kThreadsTc = 384;           // three warpgroups; warps 10 and 11 only take part in the register hand-over
 constexpr int kRegsSoftmax = 216;         // registers per thread of the softmax warpgroups after the hand-over
 constexpr int kRegsOther = 72;            // ... of the producer / MMA warpgroup
+// The CTA's register allocation is fixed at launch (65,536 / 384 threads = 170 -> 168 per thread): the softmax warps
+// can only gain what the third warpgroup gives up; a larger setmaxnreg.inc would wait forever.
+static_assert(8 * kRegsSoftmax + 4 * kRegsOther <= 12 * ((65536 / 384) / 8 * 8), "register hand-over exceeds the CTA's allocation");
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;    // log2 units: P stays below 2^8
