@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libksa_b200.so")
 KSA_OK = 0
 KSA_ERR_INVALID_ARG, KSA_ERR_UNSUPPORTED, KSA_ERR_WORKSPACE = -1, -2, -3
 KSA_ERR_CUDA, KSA_ERR_TIMEOUT, KSA_ERR_NOMEM = -4, -5, -6
+KSA_PREP_NO_ROPE = 1
 KSA_FLAG_SUMMARY_TEXT_ONLY = 0x1
 KSA_FLAG_REFERENCE_KERNEL = 0x2
 KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
@@ -33,6 +34,7 @@ EXPORTS = [
     "ksa_strerror",
     "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
     "ksa_decode_text", "ksa_decode_summary",
+    "ksa_anneal_lambda", "ksa_position_ids", "ksa_total_summary_rows", "ksa_qkv_prepare",
 ]
 
 
@@ -101,6 +103,11 @@ def lib():
     L.ksa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, pp, vp]
     L.ksa_bwd_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
+    L.ksa_anneal_lambda.argtypes = [i64, i64, i64, ctypes.POINTER(ctypes.c_float)]
+    L.ksa_position_ids.argtypes = [pp, vp]
+    L.ksa_total_summary_rows.restype = i64
+    L.ksa_total_summary_rows.argtypes = [pp]
+    L.ksa_qkv_prepare.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, pp, vp]
     L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
     L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.ksa_clear_device_status.argtypes = [vp]
@@ -199,6 +206,26 @@ def bwd_workspace_bytes(prob: Problem) -> int:
     return int(n.value)
 
 
+def anneal_lambda(step: int, s_start: int, s_end: int) -> float:
+    lam = ctypes.c_float()
+    _check(lib().ksa_anneal_lambda(step, s_start, s_end, ctypes.byref(lam)), "ksa_anneal_lambda")
+    return float(lam.value)
+
+
+def position_ids(prob: Problem):
+    """Position id of every augmented row (numpy int32), computed by the library on the host."""
+    import numpy as np
+    p = prob.params()
+    out = np.zeros(total_aug_len(prob), dtype=np.int32)
+    _check(lib().ksa_position_ids(ctypes.byref(p), out.ctypes.data), "ksa_position_ids")
+    return out
+
+
+def total_summary_rows(prob: Problem) -> int:
+    p = prob.params()
+    return int(lib().ksa_total_summary_rows(ctypes.byref(p)))
+
+
 def host_staging_bytes(prob: Problem) -> int:
     p = prob.params()
     n = ctypes.c_size_t()
@@ -265,6 +292,22 @@ class Context:
         _check(lib().ksa_attn_bwd(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                   dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), ctypes.byref(p), stream), "ksa_attn_bwd")
+
+    def qkv_prepare(self, prob: Problem, q_main, k_main, v_main, q_summ, k_summ, v_summ, q_out, k_out, v_out,
+                    lam: float, rope_theta: float, flags: int = 0, stream: Optional[int] = None):
+        """ksa_qkv_prepare on torch CUDA tensors (outputs laid out like their _main inputs; summ tensors may be None)."""
+        import torch
+        p = prob.params(q_main, k_main, v_main, q_main)
+        assert q_out.stride() == q_main.stride() and k_out.stride() == k_main.stride() and v_out.stride() == v_main.stride()
+        for t in (q_summ, k_summ, v_summ):
+            assert t is None or t.is_contiguous()
+        if stream is None:
+            stream = torch.cuda.current_stream(q_main.device).cuda_stream
+        ptr = lambda t: None if t is None else t.data_ptr()
+        _check(lib().ksa_qkv_prepare(self.handle, q_main.data_ptr(), k_main.data_ptr(), v_main.data_ptr(),
+                                     ptr(q_summ), ptr(k_summ), ptr(v_summ), q_out.data_ptr(), k_out.data_ptr(), v_out.data_ptr(),
+                                     ctypes.c_float(lam), ctypes.c_float(rope_theta), ctypes.c_uint32(flags),
+                                     ctypes.byref(p), stream), "ksa_qkv_prepare")
 
     def attn_fwd_host(self, prob: Problem, q, k, v, out, lse, staging, stream: Optional[int] = None):
         """ksa_attn_fwd_host: q, k, v, out, lse are contiguous HOST tensors (pinned recommended)."""

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "../../include/ksa.h"
+#include "../../include/ksa_prep.h"
 #include "ksa_host.h"
 #include "ksa_bwd.h"
 #include "ksa_launch.h"
@@ -114,7 +115,7 @@ void build_layout(const ksa_params* p, HostSchedule& hs)
 {
     const int k = p->chunk_len, m = p->summaries_per_chunk;
     hs.seqs.resize(p->num_seqs);
-    int64_t aug = 0, trow = 0, srow = 0;
+    int64_t aug = 0, trow = 0, srow = 0, summ_before = 0;
     hs.max_text_pad = hs.max_summ_pad = hs.max_n_summ = 0;
     for (int b = 0; b < p->num_seqs; ++b) {
         SeqInfo& s = hs.seqs[b];
@@ -124,6 +125,8 @@ void build_layout(const ksa_params* p, HostSchedule& hs)
         s.n_summ = s.n_chunks * m;
         s.aug_off = aug;
         s.chunk0 = (int32_t)(aug / (k + m));
+        s.summ_base = (int32_t)summ_before;
+        summ_before += s.n_summ;
         s.text_off = (int32_t)trow;
         s.summ_off = (int32_t)srow;
         s.text_pad = (int32_t)round_up(s.n_text, kTileM);
@@ -788,6 +791,81 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     }
     if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += (direct ? 4 : 5) + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
+    return KSA_OK;
+}
+
+// ---- Q/K/V preparation upstream of the attention (include/ksa_prep.h) --------------------------------
+extern "C" __attribute__((visibility("default"))) int ksa_anneal_lambda(int64_t step, int64_t s_start, int64_t s_end, float* lambda)
+{
+    if (!lambda || s_end <= s_start) return KSA_ERR_INVALID_ARG;
+    if (step <= s_start) *lambda = 1.f;
+    else if (step >= s_end) *lambda = 0.f;
+    else *lambda = (float)(1.0 - (double)(step - s_start) / (double)(s_end - s_start));
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int64_t ksa_total_summary_rows(const ksa_params* p)
+{
+    if (validate(p) != KSA_OK) return KSA_ERR_INVALID_ARG;
+    int64_t total = 0;
+    for (int b = 0; b < p->num_seqs; ++b)
+        total += (int64_t)((p->cu_text_lens[b + 1] - p->cu_text_lens[b]) / p->chunk_len) * p->summaries_per_chunk;
+    return total;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_position_ids(const ksa_params* p, int32_t* position_ids)
+{
+    if (!position_ids) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    const int k = p->chunk_len, m = p->summaries_per_chunk;
+    int64_t row = 0;
+    for (int b = 0; b < p->num_seqs; ++b) {
+        const int n = p->cu_text_lens[b + 1] - p->cu_text_lens[b];
+        for (int i = 0; i < n; ++i) {
+            position_ids[row++] = i;                                     // a text token keeps its index
+            if ((i + 1) % k == 0)                                        // chunk complete: its summary tokens
+                for (int r = 0; r < m; ++r) position_ids[row++] = i;     // ... take its last text token's id (Sec. 2.2.1)
+        }
+    }
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_qkv_prepare(ksa_ctx* ctx, const void* q_main, const void* k_main, const void* v_main,
+                               const void* q_summ, const void* k_summ, const void* v_summ,
+                               void* q_out, void* k_out, void* v_out, float lambda, float rope_theta, uint32_t prep_flags,
+                               const ksa_params* p, void* cuda_stream)
+{
+    if (!ctx || !q_main || !k_main || !v_main || !q_out || !k_out || !v_out) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = validate_strides(p)) != KSA_OK) return rc;
+    if (!(lambda >= 0.f && lambda <= 1.f)) return KSA_ERR_INVALID_ARG;
+    const bool rope = !(prep_flags & KSA_PREP_NO_ROPE);
+    if (rope && !(rope_theta > 0.f)) return KSA_ERR_INVALID_ARG;
+    const bool need_summ = lambda != 0.f && ksa_total_summary_rows(p) > 0;
+    if (need_summ && (!q_summ || !k_summ || !v_summ)) return KSA_ERR_INVALID_ARG;
+    const uintptr_t ptrs[9] = {(uintptr_t)q_main, (uintptr_t)k_main, (uintptr_t)v_main, (uintptr_t)q_summ, (uintptr_t)k_summ,
+                               (uintptr_t)v_summ, (uintptr_t)q_out, (uintptr_t)k_out, (uintptr_t)v_out};
+    for (int i = 0; i < 9; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
+    if ((rc = ensure_schedule(ctx, p, true)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    PrepArgs a{};
+    a.seqs = ctx->d_seqs;
+    a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.rope = rope ? 1 : 0;
+    a.lambda = need_summ ? lambda : 0.f;
+    a.log2_theta = rope ? std::log2((double)rope_theta) : 0.0;
+    a.qm = (const uint16_t*)q_main; a.km = (const uint16_t*)k_main; a.vm = (const uint16_t*)v_main;
+    a.qs = (const uint16_t*)q_summ; a.ks = (const uint16_t*)k_summ; a.vs = (const uint16_t*)v_summ;
+    a.qo = (uint16_t*)q_out; a.ko = (uint16_t*)k_out; a.vo = (uint16_t*)v_out;
+    a.q_st = p->q_stride_tok; a.q_sh = p->q_stride_head; a.k_st = p->k_stride_tok; a.k_sh = p->k_stride_head;
+    a.v_st = p->v_stride_tok; a.v_sh = p->v_stride_head;
+    int64_t max_aug_len = 0;
+    for (const SeqInfo& s : hs.seqs) max_aug_len = std::max<int64_t>(max_aug_len, (int64_t)s.n_text + s.n_summ);
+    cudaError_t e = launch_prep(a, max_aug_len, p->num_seqs, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
     return KSA_OK;
 }
 

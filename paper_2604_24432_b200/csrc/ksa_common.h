@@ -18,6 +18,7 @@ struct SeqInfo {
     int32_t text_pad;   // padded text rows (multiple of kTileM)
     int32_t summ_pad;   // padded summary rows (multiple of kTileN)
     int32_t chunk0;     // aug_off / (k + m): first chunk of the sequence in the direct views (valid if every length is a multiple of k)
+    int32_t summ_base;  // summary rows of the sequences before this one (unpadded count)
 };
 
 // One unit of work of the text-row kernel: one query tile, one or two query heads that

@@ -27,4 +27,19 @@ cudaError_t launch_text_tc(const KernelArgs& a, const TextMaps& maps, int num_sm
 // One-time per-device setup (dynamic shared memory opt-in).
 cudaError_t setup_text_tc();
 
+// Q/K/V preparation upstream of the attention (position ids, interpolation at summary positions, rotary
+// embedding): one pass over the augmented rows.
+struct PrepArgs {
+    const SeqInfo* seqs;
+    int32_t k, m, Hq, Hkv, D;
+    int32_t rope;                  // 0: interpolate only
+    float lambda;
+    double log2_theta;
+    const uint16_t* qm; const uint16_t* km; const uint16_t* vm;     // projections with the shared weights
+    const uint16_t* qs; const uint16_t* ks; const uint16_t* vs;     // ... with the summary weights, [S, H, D]
+    uint16_t* qo; uint16_t* ko; uint16_t* vo;
+    int64_t q_st, q_sh, k_st, k_sh, v_st, v_sh;
+};
+cudaError_t launch_prep(const PrepArgs& a, int64_t max_aug_len, int num_seqs, cudaStream_t stream);
+
 }  // namespace ksa
