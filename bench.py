@@ -464,6 +464,60 @@ def run_backward(args):
     return 0
 
 
+def run_prep(args):
+    """Secondary line: the Q/K/V preparation pass (position ids, interpolation at summary positions, rotary
+    embedding) over the workload's q, k, v; HBM-bound, reported as algorithmic bytes per second."""
+    from paper_2604_24432_b200 import binding as ksa
+    from paper_2604_24432_b200 import build as ksa_build
+    rank, world, local = dist_env()
+    if rank != 0:
+        return 0
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ksa_build.build()
+    wl, layout = workload_and_layout(args)
+    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total, S = ksa.total_aug_len(prob), ksa.total_summary_rows(prob)
+    qh, kh, vh = synth.make_qkv(wl, total)
+    q, k, v = qh.to(dev), kh.to(dev), vh.to(dev)
+    del qh, kh, vh
+    g = torch.Generator(device=dev).manual_seed(3)
+    mk = lambda H: torch.randn((max(S, 1), H, wl.D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    qs, ks, vs = mk(wl.Hq), mk(wl.Hkv), mk(wl.Hkv)
+    qo, ko, vo = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ctx = ksa.Context(local)
+    lam, theta = 0.5, 1.0e6                  # mid-way through the annealing window; Table 3's base after the 8K stage
+    stream = torch.cuda.current_stream(dev)
+    for _ in range(max(args.warmup, 3)):
+        ctx.qkv_prepare(prob, q, k, v, qs, ks, vs, qo, ko, vo, lam, theta)
+    torch.cuda.synchronize()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record(stream)
+        for _ in range(args.steps):
+            ctx.qkv_prepare(prob, q, k, v, qs, ks, vs, qo, ko, vo, lam, theta)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    row_bytes = (wl.Hq + 2 * wl.Hkv) * wl.D * 2
+    alg_bytes = (2 * total + S) * row_bytes          # every row read and written once, summary projections read once
+    peaks = load_peaks()
+    gbs = alg_bytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": "KSA q/k/v preparation, augmented tokens/s", "value": total / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)", "config": base_config(wl, layout, 1),
+        "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": f"of {peaks['source']} (copy bandwidth)", "kernel": "ksa_prep_kernel",
+                     "algorithmic_bytes_per_launch": alg_bytes},
+        "e2e": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def summary_pairs(wl, layout):
     """Visible pairs of the summary rows (they run in their own small kernel)."""
     tot = 0
@@ -489,6 +543,7 @@ def main():
     ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
     ap.add_argument("--decode-batch", type=int, default=32)
     ap.add_argument("--backward", action="store_true", help="secondary line: the backward pass")
+    ap.add_argument("--prep", action="store_true", help="secondary line: the q/k/v preparation pass upstream of the attention")
     ap.add_argument("--no-graph", action="store_true", help="decode: plain launches instead of a replayed CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -497,6 +552,8 @@ def main():
         return run_decode(args)
     if args.backward:
         return run_backward(args)
+    if args.prep:
+        return run_prep(args)
     return run_ours(args)
 
 
