@@ -464,6 +464,10 @@ def run_backward(args):
     return 0
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one ksa_prep_kernel launch (ncu; see profiles/)
+NCU_PREP_KERNEL_DRAM_BYTES = {("128k", "P"): 3.148e9}
+
+
 def run_prep(args):
     """Secondary line: the Q/K/V preparation pass (position ids, interpolation at summary positions, rotary
     embedding) over the workload's q, k, v; HBM-bound, reported as algorithmic bytes per second."""
@@ -510,7 +514,8 @@ def run_prep(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)", "config": base_config(wl, layout, 1),
         "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                     "traffic": None, "peak_source": f"of {peaks['source']} (copy bandwidth)", "kernel": "ksa_prep_kernel",
+                     "traffic": NCU_PREP_KERNEL_DRAM_BYTES.get((wl.name, layout.name)),
+                     "peak_source": f"of {peaks['source']} (copy bandwidth)", "kernel": "ksa_prep_kernel",
                      "algorithmic_bytes_per_launch": alg_bytes},
         "e2e": None, "cpu_baseline": None,
     }
