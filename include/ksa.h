@@ -147,6 +147,24 @@ int ksa_attn_fwd(ksa_ctx* ctx, const void* q, const void* k, const void* v,
                  void* out, float* lse, void* workspace, size_t workspace_bytes,
                  const ksa_params* p, void* cuda_stream);
 
+/* ---- sequence-parallel parts ----------------------------------------------------------- */
+/*
+ * The same operator on a contiguous part of the query rows only, so that num_parts processes (one per
+ * GPU) can share one long batch: part `part` (0 .. num_parts - 1) computes the rows
+ * [*aug_begin, *aug_end) that ksa_part_rows reports -- contiguous, in order, disjoint, covering every
+ * row, and cut so that the parts carry about the same number of visible tiles (under Eq. 3 later
+ * rows cost more).  A text row only attends to rows at or before its own and a summary row to
+ * its own chunk, so the call needs q for its own rows and k, v for the rows [0, *aug_end) -- the
+ * exchange step of a sequence-parallel run is an all-gather of k and v (or a gather from the lower
+ * ranks).  Tensors, layouts, workspace and errors are those of ksa_attn_fwd (full-size tensors,
+ * indexed by global augmented row; rows of out / lse outside the part are not touched; rows of k, v
+ * after *aug_end must hold finite values).
+ */
+int ksa_part_rows(ksa_ctx* ctx, const ksa_params* p, int32_t part, int32_t num_parts, int64_t* aug_begin, int64_t* aug_end);
+int ksa_attn_fwd_part(ksa_ctx* ctx, const void* q, const void* k, const void* v, void* out, float* lse,
+                      void* workspace, size_t workspace_bytes, const ksa_params* p, int32_t part, int32_t num_parts,
+                      void* cuda_stream);
+
 /* ---- backward ----------------------------------------------------------------------- */
 /* Bytes of DEVICE workspace ksa_attn_bwd needs for this problem. */
 int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);

@@ -35,6 +35,7 @@ EXPORTS = [
     "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
     "ksa_decode_text", "ksa_decode_summary",
     "ksa_anneal_lambda", "ksa_position_ids", "ksa_total_summary_rows", "ksa_qkv_prepare",
+    "ksa_part_rows", "ksa_attn_fwd_part",
 ]
 
 
@@ -103,6 +104,8 @@ def lib():
     L.ksa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, pp, vp]
     L.ksa_bwd_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
+    L.ksa_part_rows.argtypes = [vp, pp, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    L.ksa_attn_fwd_part.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, i32, i32, vp]
     L.ksa_anneal_lambda.argtypes = [i64, i64, i64, ctypes.POINTER(ctypes.c_float)]
     L.ksa_position_ids.argtypes = [pp, vp]
     L.ksa_total_summary_rows.restype = i64
@@ -292,6 +295,23 @@ class Context:
         _check(lib().ksa_attn_bwd(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                   dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), ctypes.byref(p), stream), "ksa_attn_bwd")
+
+    def part_rows(self, prob: Problem, part: int, num_parts: int):
+        """Augmented row range [begin, end) of part `part` of `num_parts` (ksa_part_rows)."""
+        p = prob.params()
+        b, e = ctypes.c_int64(), ctypes.c_int64()
+        _check(lib().ksa_part_rows(self.handle, ctypes.byref(p), part, num_parts, ctypes.byref(b), ctypes.byref(e)), "ksa_part_rows")
+        return int(b.value), int(e.value)
+
+    def attn_fwd_part(self, prob: Problem, q, k, v, out, lse, workspace, part: int, num_parts: int, stream: Optional[int] = None):
+        """ksa_attn_fwd_part on torch CUDA tensors: only the query rows of the part are computed."""
+        import torch
+        p = prob.params(q, k, v, out)
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        _check(lib().ksa_attn_fwd_part(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                       workspace.data_ptr(), workspace.numel() * workspace.element_size(), ctypes.byref(p),
+                                       part, num_parts, stream), "ksa_attn_fwd_part")
 
     def qkv_prepare(self, prob: Problem, q_main, k_main, v_main, q_summ, k_summ, v_summ, q_out, k_out, v_out,
                     lam: float, rope_theta: float, flags: int = 0, stream: Optional[int] = None):

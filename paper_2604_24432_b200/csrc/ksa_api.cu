@@ -665,6 +665,100 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
     return KSA_OK;
 }
 
+// ---- sequence-parallel parts ---------------------------------------------------------------------
+// The query rows are cut into num_parts contiguous parts of about equal work (Eq. 3 makes later rows more
+// expensive): the row chunks of a schedule with 16 chunks per part, grouped by their tile counts.
+static constexpr int kPartChunkFactor = 16;
+static void part_chunk_range(const HostSchedule& hs, int part, int num_parts, size_t& c0, size_t& c1)
+{
+    const size_t n = hs.chunks.size();
+    std::vector<int64_t> before(n + 1, 0);                               // tile visits of the chunks before chunk c
+    for (size_t c = 0; c < n; ++c) {
+        int64_t cost = 0;
+        for (int64_t w = hs.chunks[c].work_off; w < hs.chunks[c].work_off + hs.chunks[c].work_cnt; ++w) {
+            const WorkItem& it = hs.work[(size_t)w];
+            cost += (int64_t)it.n_heads * (it.ns_tiles + it.band_hi - it.band_lo + 1);
+        }
+        before[c + 1] = before[c] + cost;
+    }
+    auto boundary = [&](int i) -> size_t {                               // first chunk with at least i / num_parts of the work before it
+        if (i <= 0) return 0;
+        if (i >= num_parts) return n;
+        const int64_t want = (before[n] * i + num_parts - 1) / num_parts;
+        return (size_t)(std::lower_bound(before.begin(), before.end(), want) - before.begin());
+    };
+    c0 = std::min(boundary(part), n);
+    c1 = std::min(std::max(boundary(part + 1), c0), n);
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_part_rows(ksa_ctx* ctx, const ksa_params* p, int32_t part, int32_t num_parts,
+                             int64_t* aug_begin, int64_t* aug_end)
+{
+    if (!ctx || !aug_begin || !aug_end || num_parts < 1 || part < 0 || part >= num_parts) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = ensure_schedule(ctx, p, false, num_parts * kPartChunkFactor)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    size_t c0, c1;
+    part_chunk_range(hs, part, num_parts, c0, c1);
+    if (c0 == c1) {                                                      // empty part: an empty range at its place in the order
+        *aug_begin = *aug_end = (c0 < hs.chunks.size()) ? hs.chunks[c0].aug0 : hs.total_aug;
+        return KSA_OK;
+    }
+    *aug_begin = hs.chunks[c0].aug0;
+    *aug_end = hs.chunks[c1 - 1].aug1;
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_part(ksa_ctx* ctx, const void* q, const void* k, const void* v, void* out, float* lse,
+                                 void* workspace, size_t workspace_bytes, const ksa_params* p, int32_t part,
+                                 int32_t num_parts, void* cuda_stream)
+{
+    if (!ctx || !q || !k || !v || !out || !lse || num_parts < 1 || part < 0 || part >= num_parts) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = validate_strides(p)) != KSA_OK) return rc;
+    const uintptr_t ptrs[5] = {(uintptr_t)q, (uintptr_t)k, (uintptr_t)v, (uintptr_t)out, (uintptr_t)lse};
+    for (int i = 0; i < 5; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
+    if ((rc = ensure_schedule(ctx, p, true, num_parts * kPartChunkFactor)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    const bool direct = direct_ok(p);
+    const WorkspaceLayout wl = workspace_layout(p, hs);
+    if (!direct && (!workspace || workspace_bytes < wl.total || ((uintptr_t)workspace & 255))) return KSA_ERR_WORKSPACE;
+    size_t c0, c1;
+    part_chunk_range(hs, part, num_parts, c0, c1);
+    if (c0 == c1) return KSA_OK;
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    KernelArgs a = make_args(ctx, p, q, k, v, out, lse, workspace, wl, direct);
+    cudaError_t e;
+    if (!direct) {
+        // the packed streams of the whole batch (rows after the part's last row are never read unmasked, but
+        // packing them all keeps every tile finite)
+        if ((e = launch_pack(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
+    const WorkItem* work_base = a.work;
+    int64_t work_cnt = 0;
+    for (size_t ci = c0; ci < c1; ++ci) {
+        const RowChunk& c = hs.chunks[ci];
+        work_cnt += c.work_cnt;
+        if (a.m > 0 && c.summq1 > c.summ0) {                             // the summary rows whose chunks end inside this row chunk
+            a.r_seq = c.seq;
+            a.r_text0 = c.text0; a.r_text1 = c.text1;
+            a.r_summ0 = c.summ0; a.r_summ1 = c.summ1; a.r_summq1 = c.summq1;
+            if ((e = launch_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+            ctx->launches += 1;
+        }
+    }
+    a.r_seq = -1;
+    a.work = work_base + hs.chunks[c0].work_off;                         // the chunks' items follow one another in the list
+    a.num_work = (int32_t)work_cnt;
+    TextMaps maps;
+    if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
+    return launch_text(ctx, a, p->flags, maps, stream);
+}
+
 // Number of row chunks the host entry point aims for (upload / compute / download stages).
 static constexpr int kHostPipelineChunks = 8;
 

@@ -23,6 +23,49 @@ def visible_pairs_of_sequence(n: int, k: int, m: int, C: int) -> int:
     return total
 
 
+def visible_pairs_of_rows(n: int, k: int, m: int, C: int, aug_begin: int, aug_end: int) -> int:
+    """Visible (query, key) pairs of the augmented rows [aug_begin, aug_end) of one sequence of n text tokens and
+    one head: text rows by Eq. 3, summary rows their own chunk with self visibility."""
+    total = 0
+    s = k + m
+    full = (n // k) * s
+    for a in range(aug_begin, aug_end):
+        if a < full and a % s >= k:                        # summary row r of its chunk
+            total += k + (a % s - k) + 1
+            continue
+        i = (a // s) * k + a % s if a < full else (n // k) * k + (a - full)
+        c = i // k
+        far = max(0, c - C)
+        total += i - far * k + 1 + far * m
+    return total
+
+
+def kv_rows_needed(aug_end: int) -> range:
+    """Rows of k and v a sequence-parallel rank needs for query rows that end at aug_end (exclusive): a text row
+    attends to rows at or before its own, a summary row to its own chunk, so everything before aug_end and
+    nothing after it.  (Rows of the window's far side that only summaries cover could be skipped as well; the
+    all-gather below does not bother.)"""
+    return range(0, aug_end)
+
+
+def all_gather_rows(local_rows, ranges, total_rows):
+    """The exchange step of a sequence-parallel run: every rank contributes its rows [begin, end) of k (or v) and
+    receives the whole tensor.  `local_rows`: this rank's [end - begin, H, D] tensor; `ranges`: the (begin, end)
+    of every rank, in rank order.  Uses one all_gather over equally sized (padded) buffers."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size()
+    longest = max(e - b for b, e in ranges)
+    pad = torch.zeros((longest,) + tuple(local_rows.shape[1:]), dtype=local_rows.dtype, device=local_rows.device)
+    pad[:local_rows.shape[0]] = local_rows
+    parts = [torch.empty_like(pad) for _ in range(world)]
+    dist.all_gather(parts, pad)
+    full = torch.zeros((total_rows,) + tuple(local_rows.shape[1:]), dtype=local_rows.dtype, device=local_rows.device)
+    for (b, e), t in zip(ranges, parts):
+        full[b:e] = t[:e - b]
+    return full
+
+
 def shard_sequences(text_lens: Sequence[int], k: int, m: int, C: int, world: int) -> List[List[int]]:
     """Indices of the sequences each rank processes (every sequence exactly once): longest first onto
     the least loaded rank; ties go to the lower rank, so every rank computes the same table."""

@@ -71,3 +71,69 @@ def test_shards_are_balanced_and_head_ranges_tile():
         assert max(loads) - min(loads) <= max(cost)          # longest-first never does worse than one item
         ranges = dist_utils.shard_kv_heads(8, world)
         assert [h for r in ranges for h in r] == list(range(8))
+
+
+def _split_rows_by_work(n, k, m, C, world):
+    """Contiguous augmented row ranges of about equal visible pairs (what the library's ksa_part_rows does at tile
+    granularity; here row by row, for the CPU test)."""
+    L = orc.aug_len(n, k, m)
+    cost = [dist_utils.visible_pairs_of_rows(n, k, m, C, a, a + 1) for a in range(L)]
+    total, acc, cuts = sum(cost), 0, [0]
+    for a, c in enumerate(cost):
+        acc += c
+        while len(cuts) < world and acc * world >= total * len(cuts):
+            cuts.append(a + 1)
+    cuts += [L] * (world + 1 - len(cuts))
+    return [(cuts[r], cuts[r + 1]) for r in range(world)]
+
+
+def _seq_parallel_worker(rank, world, port, ret):
+    """Sequence-parallel forward over gloo: every rank owns a part of the rows of one sequence, contributes its rows
+    of k and v to an all-gather, computes its own query rows (here with the oracle standing in for the kernel:
+    it only reads k, v rows before the part's end) and the parts together equal the whole."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        n, k, m, C, Hq, Hkv, D = 150, 8, 1, 3, 2, 1, 16
+        wl = synth.Workload("sp", 5, [n], Hq, Hkv, D)
+        L = orc.aug_len(n, k, m)
+        q, kk, v = synth.make_qkv(wl, L)                     # every rank draws the same tensors ...
+        ranges = _split_rows_by_work(n, k, m, C, world)
+        b, e = ranges[rank]
+        k_full = dist_utils.all_gather_rows(kk[b:e].clone(), ranges, L)     # ... but only contributes its own rows
+        v_full = dist_utils.all_gather_rows(v[b:e].clone(), ranges, L)
+        assert torch.equal(k_full, kk) and torch.equal(v_full, v)
+        # what the rank may look at: its own q rows, k and v before the end of its part (Eq. 3)
+        need = dist_utils.kv_rows_needed(e)
+        k_loc, v_loc = torch.zeros_like(kk), torch.zeros_like(v)
+        k_loc[need.start:need.stop] = k_full[need.start:need.stop]
+        v_loc[need.start:need.stop] = v_full[need.start:need.stop]
+        rows = list(range(b, e))
+        out_part, lse_part, _ = orc.fwd(synth.bits(q), synth.bits(k_loc), synth.bits(v_loc), [n], k, m, C, wl.scale, rows=rows)
+        out_ref, lse_ref, _ = orc.fwd(synth.bits(q), synth.bits(kk), synth.bits(v), [n], k, m, C, wl.scale, rows=rows)
+        assert (out_part == out_ref).all() and (lse_part == lse_ref).all()
+        # the parts tile the rows and carry about the same work
+        work = [dist_utils.visible_pairs_of_rows(n, k, m, C, x, y) for x, y in ranges]
+        assert sum(work) == dist_utils.visible_pairs_of_sequence(n, k, m, C)
+        assert ranges[0][0] == 0 and ranges[-1][1] == L and all(r0[1] == r1[0] for r0, r1 in zip(ranges, ranges[1:]))
+        assert max(work) <= 1.25 * sum(work) / world
+        ret[rank] = "ok"
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_sequence_parallel_exchange():
+    port = _free_port()
+    mgr = mp.Manager()
+    ret = mgr.dict()
+    mp.spawn(_seq_parallel_worker, args=(2, port, ret), nprocs=2, join=True)
+    assert dict(ret) == {0: "ok", 1: "ok"}
+
+
+def test_row_costs_add_up_to_the_oracle_pair_count():
+    for n, k, m, C in [(100, 8, 1, 2), (37, 4, 2, 0), (130, 64, 8, 1)]:
+        L = orc.aug_len(n, k, m)
+        for a in (0, 1, L // 2, L - 1):
+            assert dist_utils.visible_pairs_of_rows(n, k, m, C, a, a + 1) == orc.visible_count(n, k, m, C, a)
+        assert dist_utils.visible_pairs_of_rows(n, k, m, C, 0, L) == dist_utils.visible_pairs_of_sequence(n, k, m, C)
