@@ -468,6 +468,83 @@ def run_backward(args):
 NCU_PREP_KERNEL_DRAM_BYTES = {("128k", "P"): 3.148e9}
 
 
+def run_seq_parallel(args):
+    """Secondary line (--seq-parallel): ONE batch shared by all ranks.  Every rank owns a work-balanced part of the
+    query rows (ksa_part_rows); a step is the exchange (all-gather of the ranks' rows of k and v over NCCL) plus the
+    part's attention.  Total work is fixed as N grows: "scaling": "strong"."""
+    from paper_2604_24432_b200 import binding as ksa
+    from paper_2604_24432_b200 import build as ksa_build
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    ksa_build.build()
+    wl, layout = workload_and_layout(args)
+    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total = ksa.total_aug_len(prob)
+    flops = 4.0 * wl.D * wl.Hq * ksa.visible_pairs(prob)
+    ctx = ksa.Context(local)
+    ranges = [ctx.part_rows(prob, r, world) for r in range(world)]
+    b, e = ranges[rank]
+    qh, kh, vh = synth.make_qkv(wl, total)               # the same batch on every rank; a rank keeps its own rows only
+    q = torch.zeros((total, wl.Hq, wl.D), dtype=torch.bfloat16, device=dev)
+    q[b:e] = qh[b:e].to(dev)
+    k_mine, v_mine = kh[b:e].to(dev), vh[b:e].to(dev)
+    del qh, kh, vh
+    out = torch.empty((total, wl.Hq, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        if world > 1:
+            k_full = dist_utils.all_gather_rows(k_mine, ranges, total)
+            v_full = dist_utils.all_gather_rows(v_mine, ranges, total)
+        else:
+            k_full, v_full = k_mine, v_mine
+        ctx.attn_fwd_part(prob, q, k_full, v_full, out, lse, ws, rank, world)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+    assert ctx.device_status() == 0
+    ms = dist_utils.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+    if rank == 0:
+        peaks = load_peaks()
+        val = flops / (ms * 1e-3) / 1e12
+        cfg = base_config(wl, layout, 1)
+        cfg["parallelism"] = f"sequence parallel x{world}: rows [{b}, {e}) of {total} on rank 0, all-gather of k and v per step"
+        print(json.dumps({
+            "metric": "KSA attn fwd visible TFLOP/s, one batch shared by all ranks", "value": val, "unit": "TFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)", "config": cfg,
+            "clocks": clocks.summary(), "gpu_launches": int(ctx.launch_count() - launches0),
+            "roofline": {"bound": "tensor", "achieved": val, "peak": world * peaks["bf16_sustained"], "unit": "TFLOP/s",
+                         "frac": val / (world * peaks["bf16_sustained"]), "traffic": None,
+                         "peak_source": f"of {peaks['source']} (sustained bf16 GEMM x {world})", "kernel": "ksa_text_tc_kernel (whole step incl. exchange)"},
+            "e2e": None, "cpu_baseline": None}))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
 def run_prep(args):
     """Secondary line: the Q/K/V preparation pass (position ids, interpolation at summary positions, rotary
     embedding) over the workload's q, k, v; HBM-bound, reported as algorithmic bytes per second."""
@@ -548,6 +625,8 @@ def main():
     ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
     ap.add_argument("--decode-batch", type=int, default=32)
     ap.add_argument("--backward", action="store_true", help="secondary line: the backward pass")
+    ap.add_argument("--seq-parallel", action="store_true",
+                    help="secondary line: one batch shared by all ranks (work-balanced row parts, all-gather of k and v)")
     ap.add_argument("--prep", action="store_true", help="secondary line: the q/k/v preparation pass upstream of the attention")
     ap.add_argument("--no-graph", action="store_true", help="decode: plain launches instead of a replayed CUDA graph")
     args = ap.parse_args()
@@ -559,6 +638,8 @@ def main():
         return run_backward(args)
     if args.prep:
         return run_prep(args)
+    if args.seq_parallel:
+        return run_seq_parallel(args)
     return run_ours(args)
 
 
