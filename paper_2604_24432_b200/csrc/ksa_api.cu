@@ -949,7 +949,8 @@ extern "C" __attribute__((visibility("default"))) int ksa_qkv_prepare(ksa_ctx* c
     a.k = p->chunk_len; a.m = p->summaries_per_chunk; a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
     a.rope = rope ? 1 : 0;
     a.lambda = need_summ ? lambda : 0.f;
-    a.log2_theta = rope ? std::log2((double)rope_theta) : 0.0;
+    for (int d = 0; d < p->head_dim / 2 && d < 64; ++d)
+        a.inv_freq[d] = rope ? std::pow((double)rope_theta, -2.0 * d / (double)p->head_dim) : 0.0;
     a.qm = (const uint16_t*)q_main; a.km = (const uint16_t*)k_main; a.vm = (const uint16_t*)v_main;
     a.qs = (const uint16_t*)q_summ; a.ks = (const uint16_t*)k_summ; a.vs = (const uint16_t*)v_summ;
     a.qo = (uint16_t*)q_out; a.ko = (uint16_t*)k_out; a.vo = (uint16_t*)v_out;

@@ -34,7 +34,7 @@ struct PrepArgs {
     int32_t k, m, Hq, Hkv, D;
     int32_t rope;                  // 0: interpolate only
     float lambda;
-    double log2_theta;
+    double inv_freq[64];           // theta^(-2 d / D), d = 0 .. D/2 - 1 (head_dim <= 128)
     const uint16_t* qm; const uint16_t* km; const uint16_t* vm;     // projections with the shared weights
     const uint16_t* qs; const uint16_t* ks; const uint16_t* vs;     // ... with the summary weights, [S, H, D]
     uint16_t* qo; uint16_t* ko; uint16_t* vo;

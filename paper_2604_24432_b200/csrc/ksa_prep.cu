@@ -2,8 +2,9 @@
 // summary positions (Sec. 4.1) and the rotary embedding, one pass, HBM-bound.
 //
 // A thread owns one augmented row and one 8-element slice d0 .. d0 + 7 of the first half of a head together
-// with its partners d0 + D/2 ..: it works out the row's position id and the eight angles once (double
-// precision: a position of 10^5 times a frequency near 1 has no fraction left in fp32) and then walks the
+// with its partners d0 + D/2 ..: it works out the row's position id and the eight angles once (the product
+// position x frequency and its reduction to [-pi, pi] in double precision: a position of 10^5 times a frequency
+// near 1 has no fraction left in fp32; the frequencies come from the host as doubles) and then walks the
 // heads of q, k and v with 16-byte loads and stores.  32 rows x D/16 slices per block, one sequence per grid.y.
 #include <cuda_runtime.h>
 
@@ -47,10 +48,11 @@ __global__ void __launch_bounds__(256) ksa_prep_kernel(PrepArgs a)
     if (a.rope) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const double inv_freq = exp2(-2.0 * (double)(d0 + e) / (double)a.D * a.log2_theta);
-            double s, c;
-            sincos((double)pos * inv_freq, &s, &c);
-            cs[e] = (float)c; sn[e] = (float)s;
+            // angle and its reduction to [-pi, pi] in double (a handful of fp64 operations), sine and cosine in fp32
+            const double ang = (double)pos * a.inv_freq[d0 + e];
+            const double turns = rint(ang * 0.15915494309189535);        // 1 / (2 pi)
+            const float r = (float)fma(-turns, 6.283185307179586, ang);
+            sincosf(r, &sn[e], &cs[e]);
         }
     }
     const bool blend = summ_index >= 0 && a.lambda != 0.f;
