@@ -62,7 +62,7 @@ static_assert(kBwdTcLayoutBytes <= kBwdTcSmem, "shared memory layout");
 
 // Optional event trace (compile with -DKSA_BWD_TRACE=1 for the dQ kernel, =3 for the dK / dV kernel over summary
 // keys): one CTA records (event id, clock) pairs for lane 0 of every row warp; ksa_debug_read_bwd_trace() copies
-// them out.
+// them out.  =2 / =4: no stamps, only the MMA issuer's waiting times (below).
 #ifdef KSA_BWD_TRACE
 constexpr int kBtEvents = 4096;
 __device__ uint2 g_btrace[17][kBtEvents];         // role 0: MMA issuer (sums only); 1 + w: row warp w
@@ -73,6 +73,15 @@ __device__ uint32_t g_btrace_cnt[17];
     } while (0)
 #else
 #define KSA_BT(role, id) do { } while (0)
+#endif
+// KSA_BWD_TRACE == 2 / 4: the MMA issuer of one CTA of the dQ / the dK/dV (summary keys) kernel sums the cycles it
+// spends waiting for the row warps (registers only, written once at the end: stamps in memory disturb the waits).
+#if defined(KSA_BWD_TRACE) && (KSA_BWD_TRACE == 2 || KSA_BWD_TRACE == 4)
+#define KSA_BT_WAIT_BEGIN() const uint32_t bt_w0 = (uint32_t)clock()
+#define KSA_BT_WAIT_END(acc) acc += (uint32_t)clock() - bt_w0
+#else
+#define KSA_BT_WAIT_BEGIN() do { } while (0)
+#define KSA_BT_WAIT_END(acc) do { } while (0)
 #endif
 
 __device__ __forceinline__ uint32_t bt_ld_shared(uint32_t addr)
@@ -319,18 +328,32 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
             if (alive) { bt_product(tY, sm.a2(), sm.b2(0)); tc_commit(sm.bar(BB_YFULL)); }
+            uint32_t bt_wait_a = 0, bt_wait_b = 0;
+            const uint32_t bt_loop0 = (uint32_t)clock();
+            (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0;
             for (int j = 0; j < J && alive; ++j) {
                 // later stages were checked by row warp 0 before its arrivals
-                if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                { KSA_BT_WAIT_BEGIN();
+                  if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                  KSA_BT_WAIT_END(bt_wait_a); }
                 tc_fence_after();
                 bt_accumulate(tDV, tX, sm.b2(j & 1), j == 0);                               // dV += P^T dO_j
                 if (j + 1 < J) { bt_product(tX, sm.a1(), sm.b1((j + 1) % kB1Stages)); tc_commit(sm.bar(BB_XFULL)); }
-                if (!bt_wait(sm.bar(BB_PB), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                { KSA_BT_WAIT_BEGIN();
+                  if (!bt_wait(sm.bar(BB_PB), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                  KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
                 bt_accumulate(tDK, tY, sm.b1(j % kB1Stages), j == 0);                       // dK += dS^T Q_j
                 if (j + 1 < J) { bt_product(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
             }
             tc_commit(sm.bar(BB_OFULL));
+#if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 4
+            if (summ && blockIdx.x == 1 && blockIdx.y == 4 && blockIdx.z == 0) {
+                g_btrace[0][0] = make_uint2(bt_wait_a, bt_wait_b);
+                g_btrace[0][1] = make_uint2((uint32_t)clock() - bt_loop0, (uint32_t)J);
+                g_btrace_cnt[0] = 2;
+            }
+#endif
         }
     } else {
         // =============================== key rows ===================================
@@ -573,23 +596,37 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
             if (alive) { bt_product(tY(0), sm.a2(), sm.b2(0)); tc_commit(y_full(0)); }
+            uint32_t bt_wait_a = 0, bt_wait_b = 0;
+            const uint32_t bt_loop0 = (uint32_t)clock();
+            (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0;
             for (int j = 0; j < J && alive; ++j) {
                 // later stages were checked by row warp 0 before its arrival
                 if (j + 1 < J) {
                     // phase A of tile j has read X into registers; the other Y buffer was read by dQ += dS K_{j-1}
+                    KSA_BT_WAIT_BEGIN();
                     if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                    KSA_BT_WAIT_END(bt_wait_a);
                     tc_fence_after();
                     bt_product(tX, sm.a1(), sm.b1((j + 1) % kB1Stages));
                     tc_commit(sm.bar(BB_XFULL));
                     bt_product(tY(j + 1), sm.a2(), sm.b2((j + 1) & 1));
                     tc_commit(y_full(j + 1));
                 }
-                if (!bt_wait(p_b(j), (j >> 1) & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                { KSA_BT_WAIT_BEGIN();
+                  if (!bt_wait(p_b(j), (j >> 1) & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                  KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
                 bt_accumulate(tDQ, tY(j), sm.b1(j % kB1Stages), j == 0);                    // dQ += dS K_j
                 tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // K_j is free after that
             }
             tc_commit(sm.bar(BB_OFULL));
+#if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 2
+            if (blockIdx.x == 8 && blockIdx.y == 0 && blockIdx.z == 0) {
+                g_btrace[0][0] = make_uint2(bt_wait_a, bt_wait_b);
+                g_btrace[0][1] = make_uint2((uint32_t)clock() - bt_loop0, (uint32_t)J);
+                g_btrace_cnt[0] = 2;
+            }
+#endif
         }
     } else {
         // =============================== query rows =================================
