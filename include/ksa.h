@@ -166,7 +166,9 @@ int ksa_attn_fwd_part(ksa_ctx* ctx, const void* q, const void* k, const void* v,
                       void* cuda_stream);
 
 /* ---- backward ----------------------------------------------------------------------- */
-/* Bytes of DEVICE workspace ksa_attn_bwd needs for this problem. */
+/* Bytes of DEVICE workspace ksa_attn_bwd needs for this problem: the fp32 accumulators of dK / dV and two fp32
+ * scalars per text row and query head, plus packed copies of q, k, v and dout unless they can be read in place
+ * (head_dim 128 and every sequence a whole number of chunks). */
 int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
 /*
  * Gradients of ksa_attn_fwd (the kernel of Sec. 2.3 is the one "for training and prefill"):

@@ -769,11 +769,13 @@ struct BwdLayout { WorkspaceLayout fwd; size_t dot, lse_t, delta_t, dkt, dvt, dk
 static BwdLayout bwd_layout(const ksa_params* p, const HostSchedule& hs)
 {
     BwdLayout b{};
-    b.fwd = workspace_layout(p, hs);
+    // no packed streams and no packed dO where the tensor-core kernels read the caller's tensors in place
+    const bool direct = p->head_dim == 128 && direct_ok(p);
+    if (!direct) b.fwd = workspace_layout(p, hs);
     size_t off = b.fwd.total;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
     const size_t D = (size_t)p->head_dim;
-    b.dot = take((size_t)p->num_q_heads * hs.text_rows * D * 2);
+    b.dot = take(direct ? 0 : (size_t)p->num_q_heads * hs.text_rows * D * 2);
     b.lse_t = take((size_t)p->num_q_heads * hs.text_rows * 4);
     b.delta_t = take((size_t)p->num_q_heads * hs.text_rows * 4);
     b.dkt = take((size_t)p->num_kv_heads * hs.text_rows * D * 4);

@@ -190,5 +190,10 @@ def test_backward_workspace_and_limits():
     extra = 8 * text_rows * 256 + 2 * 8 * text_rows * 4 + 2 * 2 * (text_rows + summ_rows) * 128 * 4
     got = ksa.bwd_workspace_bytes(prob)
     assert fwd + extra <= got <= fwd + extra + 16 * 1024
+    # whole chunks and head_dim 128: q, k, v, dout are read in place -- only the row scalars and the fp32 accumulators
+    direct = ksa.Problem([1024, 640], 8, 1, 4, 8, 2, 128, 0.088)
+    text_rows, summ_rows = 1024 + 640, 128 + 128
+    small = 2 * 8 * text_rows * 4 + 2 * 2 * (text_rows + summ_rows) * 128 * 4
+    assert small <= ksa.bwd_workspace_bytes(direct) <= small + 16 * 1024
     many = ksa.Problem([8] * 70000, 8, 1, 2, 4, 2, 64, 0.125)
     assert _status_of(lambda: ksa.workspace_bytes(many)) == ksa.KSA_ERR_UNSUPPORTED
