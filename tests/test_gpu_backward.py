@@ -123,3 +123,49 @@ def test_backward_full_size_identities(ctx, workload):
     assert (np.abs(vdv - odo) <= 2e-3 * (vabs + oabs)).all(), (vdv, odo, vabs)
     # the identities are not met by zeros only: the gradients have their expected size
     assert (qabs > 0).all() and (vabs > 0).all()
+
+
+def test_full_causal_mode_against_torch_attention(ctx):
+    """m = 0 and a window that covers every chunk reduce the operator to plain causal attention: forward and
+    backward against torch's scaled_dot_product_attention and autograd in fp32 on the same bf16 inputs (a library
+    routine, at a size the CPU oracle would need minutes for)."""
+    n, k, Hq, Hkv, D = 4096, 8, 8, 2, 128
+    G = Hq // Hkv
+    dev = torch.device("cuda", 0)
+    wl = synth.Workload("causal", 51, [n], Hq, Hkv, D)
+    prob = ksa.Problem([n], k, 0, 1 << 20, Hq, Hkv, D, wl.scale, 0)
+    q, kk, v = synth.make_qkv(wl, n)
+    g = torch.Generator("cpu").manual_seed(52)
+    dout = torch.randn((n, Hq, D), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    qd, kd, vd, gd = q.to(dev), kk.to(dev), v.to(dev), dout.to(dev)
+    out = torch.empty_like(qd); lse = torch.empty((Hq, n), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx.clear_device_status()
+    ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws)
+    dq = torch.empty_like(qd); dk = torch.empty_like(kd); dv = torch.empty_like(vd)
+    wsb = torch.empty(ksa.bwd_workspace_bytes(prob), dtype=torch.uint8, device=dev)
+    ctx.attn_bwd(prob, qd, kd, vd, out, lse, gd, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    # reference: [heads, n, D] in fp32, K / V heads repeated over their group
+    qr = qd.float().transpose(0, 1).contiguous().requires_grad_(True)
+    kr = kd.float().transpose(0, 1).contiguous().requires_grad_(True)
+    vr = vd.float().transpose(0, 1).contiguous().requires_grad_(True)
+    from torch.nn.attention import SDPBackend, sdpa_kernel
+    with sdpa_kernel(SDPBackend.MATH):
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            qr[None], kr.repeat_interleave(G, dim=0)[None], vr.repeat_interleave(G, dim=0)[None],
+            is_causal=True, scale=wl.scale)[0]
+    ref.backward(gd.float().transpose(0, 1))
+    got = out.float().transpose(0, 1)
+    assert (got - ref.detach()).abs().max().item() <= 2e-2
+    assert (got - ref.detach()).abs().mean().item() <= 2e-3
+    # natural-log LSE of the scaled scores over the visible keys, by torch
+    scores = torch.einsum("hid,hjd->hij", qr.detach(), kr.detach().repeat_interleave(G, dim=0)) * wl.scale
+    scores = scores.masked_fill(torch.ones(n, n, dtype=torch.bool, device=dev).triu(1), float("-inf"))
+    lse_ref = torch.logsumexp(scores, dim=2)
+    assert ((lse - lse_ref).abs() <= 1e-3 * lse_ref.abs().clamp(min=1.0)).all()
+    for name, mine, theirs in (("dq", dq, qr.grad), ("dk", dk, kr.grad), ("dv", dv, vr.grad)):
+        err = (mine.float().transpose(0, 1) - theirs).abs()
+        assert err.max().item() <= 2e-2 * theirs.abs().max().item() + 1e-5, name
+        assert err.mean().item() <= 1e-2 * theirs.abs().mean().item() + 1e-5, name
