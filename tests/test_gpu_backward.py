@@ -76,7 +76,7 @@ def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     _check("dv", dv.double().cpu().numpy(), rdv)
 
 
-@pytest.mark.parametrize("workload", ["32k", "128k"])
+@pytest.mark.parametrize("workload", ["32k", "128k", "varlen"])
 def test_backward_full_size_identities(ctx, workload):
     """Full-size workloads, in the launch configuration the bench times: two identities that hold for the exact
     gradients at any size and involve every element of dq, dk and dv.
