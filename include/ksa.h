@@ -197,7 +197,7 @@ int ksa_attn_bwd(ksa_ctx* ctx, const void* q, const void* k, const void* v, cons
 int ksa_host_staging_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
 /*
  * Same operator with HOST tensors (contiguous [total_aug, H, D]; strides in p are
- * ignored).  The query tiles are cut into about eight row chunks in sequence order and
+ * ignored).  The query tiles are cut into about sixteen row chunks in sequence order and
  * pipelined: while one chunk's rows of q, k, v are copied to the device staging buffer
  * (on a copy stream the context owns), the previous chunk is packed and computed on
  * cuda_stream, and the one before that has its rows of out and lse copied back (on a
