@@ -395,7 +395,10 @@ def run_decode(args):
         "clocks": clocks.summary(),
         "gpu_launches": int(launches_per_chunk * (steps // k)) if graph is not None else int(ctx.launch_count() - launches0),
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                     "traffic": None, "peak_source": f"of {peaks['source']} (copy bandwidth)",
+                     # dram__bytes_read.sum + dram__bytes_write.sum of one ksa_decode_attn_kernel launch (ncu; see profiles/),
+                     # for the default batch of 32 sequences at a 128K context
+                     "traffic": 1.137e9 if (B, ctx_len) == (32, 131072) else None,
+                     "peak_source": f"of {peaks['source']} (copy bandwidth)",
                      "kernel": "ksa_decode_attn_kernel (+ append, merge, commit)",
                      "bytes_per_step": bytes_read / steps},
         "e2e": None, "cpu_baseline": None,
