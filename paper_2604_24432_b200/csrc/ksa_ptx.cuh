@@ -1,4 +1,4 @@
-// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, no multicast),
+// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, every CTA loads for itself),
 // tcgen05 (TMEM allocation, MMA, commit, ld/st) and the UMMA descriptor encodings.
 #pragma once
 #include <cuda.h>
