@@ -6,8 +6,8 @@
 // and the row warps turn them into bf16 operands for the accumulating MMAs in two phases:
 //   phase A (after X_j)   P = exp2(X scale - lse) on the visible pairs, kept in registers
 //   phase B (after Y_j)   dS = P (Y - delta), written as bf16 over the first half of Y's own columns
-// X and Y are single buffers, yet the pipe stays busy: while the warps are in phase A of tile j + 1 it
-// runs the accumulation from Y_j and the product Y_{j+1}; while they are in phase B, the work on X.
+// With single X and Y buffers (dK / dV) the pipe still has work while the warps compute: during phase A of
+// tile j + 1 it runs the accumulation from Y_j and the product Y_{j+1}; during phase B, the work on X.
 // TMEM (512 columns): X [0,128), Y [128,256), accumulators from 256.
 //
 //   dK / dV  key-stationary and transposed: A1 = K tile, A2 = V tile (text or summary stream), B1 = Q tile,
@@ -29,8 +29,9 @@
 // warps: row warp 0 checks that the next B1 / B2 stage has landed before it arrives.  The tensor pipe
 // works in order, so the completion of a product also tells which stage the accumulation before it has
 // finished with: row warp 0, which sees every completion of X and Y, passes that on to the producer
-// through one "empty" barrier per stage (the issuer is spared the extra commits; the producer itself may
-// fall several completions behind, which a parity wait cannot follow).  Every mbarrier wait is bounded
+// through one "empty" barrier per stage (the issuer is spared the extra commits -- except for the K
+// stages of dQ, which the early products would otherwise release too late; the producer itself may fall
+// several completions behind, which a parity wait cannot follow).  Every mbarrier wait is bounded
 // (status word + CTA-wide abort flag).
 #include <cuda_bf16.h>
 
@@ -55,7 +56,7 @@ constexpr int kOffBars = kOffB2 + kB2Stages * kBwdTileBytes;                    
 constexpr int kOffMisc = kOffBars + 192;                                              // TMEM slot, abort flags
 constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [2][lse, delta][128] per-query scalars
 constexpr int kBwdTcLayoutBytes = kOffRow + 2 * 2 * 128 * 4;
-constexpr int kBwdTcSmem = 232448;              // the whole opt-in window: the layout needs all but 832 bytes of it
+constexpr int kBwdTcSmem = 232448;              // the whole opt-in window: the layout needs all but 768 bytes of it
 enum : int { BB_AFULL = 0, BB_B1FULL = 1, BB_B2FULL = 4, BB_XFULL = 6, BB_YFULL = 7, BB_PA = 8, BB_PB = 9, BB_OFULL = 10,
              BB_B1EMPTY = 11, BB_B2EMPTY = 14, BB_YFULL2 = 16, BB_PB2 = 17 };
 static_assert(kBwdTcLayoutBytes <= kBwdTcSmem, "shared memory layout");
