@@ -49,6 +49,8 @@ def _check(name, got, ref):
     ([1280], 64, 8, 4, 4, 2, 128, 0),
     ([704, 48], 16, 0, 7, 4, 4, 128, 0),
     ([640], 8, 1, 3, 4, 1, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
+    ([500], 8, 3, 2, 4, 2, 128, 0),                   # three summaries per chunk: packed streams, 128 % m != 0
+    ([400, 136], 8, 1, 2, 4, 4, 128, 0),              # one query head per KV head, with summaries
 ])
 def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
