@@ -21,6 +21,9 @@
  *   - ksa_attn_fwd is asynchronous on the given CUDA stream and performs no host
  *     synchronisation once the schedule for the given lengths is cached (the first
  *     call with a new set of lengths builds and uploads it with a blocking copy).
+ *     The same holds for ksa_attn_bwd, ksa_attn_fwd_part and ksa_qkv_prepare: after
+ *     that first call they may be recorded into a CUDA graph (stream capture) and
+ *     replayed on the same buffers.
  *   - There is no CPU fallback: on a machine without an sm_100 device ksa_create fails.
  *
  * Layout of one packed batch (Eq. 1, generalised to m summaries per chunk):
