@@ -6,16 +6,15 @@
 // and the row warps turn them into bf16 operands for the accumulating MMAs in two phases:
 //   phase A (after X_j)   P = exp2(X scale - lse) on the visible pairs, kept in registers
 //   phase B (after Y_j)   dS = P (Y - delta), written as bf16 over the first half of Y's own columns
-// With single X and Y buffers (dK / dV) the pipe still has work while the warps compute: during phase A of
-// tile j + 1 it runs the accumulation from Y_j and the product Y_{j+1}; during phase B, the work on X.
 // TMEM (512 columns): X [0,128), Y [128,256), accumulators from 256.
 //
 //   dK / dV  key-stationary and transposed: A1 = K tile, A2 = V tile (text or summary stream), B1 = Q tile,
 //            B2 = dO tile of the (query tile, query head) pairs that see the keys; X = S^T, Y = dP^T.
-//            Phase A also writes P^T as bf16 over X.  Pipe order per j: dV += P^T dO_j, X_{j+1},
-//            dK += dS^T Q_j, Y_{j+1}.  At the end each key row adds dV and scale * dK to the fp32
-//            accumulators of its stream (vector atomics: several segments and the summary-row kernel
-//            add to the same rows).
+//            The warps hand X back as soon as it is in their registers, so X_{j+1} runs beside the
+//            exponentials of tile j; phase B writes dS^T over columns 0 .. 15 and P^T over columns 16 .. 31 of
+//            each warp's 32-column block of Y.  Pipe order per j: X_{j+1}, dV += P^T dO_j, dK += dS^T Q_j,
+//            Y_{j+1}.  At the end each key row adds dV and scale * dK to the fp32 accumulators of its stream
+//            (vector atomics: several segments and the summary-row kernel add to the same rows).
 //   dQ       query-stationary: A1 = Q tile, A2 = dO tile, B1 = K tile, B2 = V tile over the visible
 //            summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP.  One accumulator leaves
 //            room for a second Y buffer (columns from 384), so both products of tile j + 1 are issued
@@ -28,11 +27,12 @@
 // producer; warp 17: MMA issuer.  The issuer's time is the critical path, so it waits only for the row
 // warps: row warp 0 checks that the next B1 / B2 stage has landed before it arrives.  The tensor pipe
 // works in order, so the completion of a product also tells which stage the accumulation before it has
-// finished with: row warp 0, which sees every completion of X and Y, passes that on to the producer
-// through one "empty" barrier per stage (the issuer is spared the extra commits -- except for the K
-// stages of dQ, which the early products would otherwise release too late; the producer itself may fall
-// several completions behind, which a parity wait cannot follow).  Every mbarrier wait is bounded
-// (status word + CTA-wide abort flag).
+// finished with: in the dQ kernel row warp 0, which sees every completion of X and Y, passes that on to
+// the producer through one "empty" barrier per stage (the issuer is spared the extra commits -- except
+// for the K stages, which the early products would otherwise release too late); in the dK / dV kernel the
+// issuer commits to the "empty" barriers right behind each accumulation.  (The producer itself may fall
+// several completions behind, which a parity wait on a shared barrier cannot follow: hence one barrier
+// per stage.)  Every mbarrier wait is bounded (status word + CTA-wide abort flag).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -272,8 +272,9 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     BtSmem sm;
     if (!bt_layout(sm, bsm_raw, a.status)) return;
     uint8_t* base_ptr = bsm_raw + (sm.base - smem_u32(bsm_raw));
-    // per-query scalars of the streamed tile, double-buffered by j: [j & 1][lse, delta][128 columns]; written by
-    // the warps of row quarter 0 (warp 4 cg writes columns 32 cg ..) one tile ahead, see below
+    // per-query scalars of the streamed tile, double-buffered by j: [j & 1][lse, delta][128 columns]; every row
+    // warp writes the 32 columns it reads itself, one tile ahead (the four warps of a column group write the same
+    // values, and each relies on its own writes only), see below
     float* rows = reinterpret_cast<float*>(base_ptr + kOffRow);
     const int quarter = warp & 3, cg = warp >> 2;                        // row warps: lanes 32 quarter ..; columns 32 cg ..
     const bool scalar_writer = warp < 16 && quarter == 0;
@@ -329,30 +330,46 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
             if (alive) { bt_product(tY, sm.a2(), sm.b2(0)); tc_commit(sm.bar(BB_YFULL)); }
-            uint32_t bt_wait_a = 0, bt_wait_b = 0;
+            uint32_t bt_wait_a = 0, bt_wait_b = 0, bt_wait_c = 0, bt_iss_x = 0, bt_iss_acc = 0;
             const uint32_t bt_loop0 = (uint32_t)clock();
-            (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0;
+            (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0; (void)bt_wait_c; (void)bt_iss_x; (void)bt_iss_acc;
             for (int j = 0; j < J && alive; ++j) {
-                // later stages were checked by row warp 0 before its arrivals
+                // the warps hold X_j in registers: the next S^T product may overwrite it while they exponentiate
                 { KSA_BT_WAIT_BEGIN();
                   if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                   KSA_BT_WAIT_END(bt_wait_a); }
                 tc_fence_after();
-                bt_accumulate(tDV, tX, sm.b2(j & 1), j == 0);                               // dV += P^T dO_j
-                if (j + 1 < J) { bt_product(tX, sm.a1(), sm.b1((j + 1) % kB1Stages)); tc_commit(sm.bar(BB_XFULL)); }
+                if (j + 1 < J) {
+                    const int s1 = (j + 1) % kB1Stages;
+                    { KSA_BT_WAIT_BEGIN();
+                    if (!bt_wait(sm.bar(BB_B1FULL + s1), ((j + 1) / kB1Stages) & 1, abort_addr, a.status, kStatusWaitQFull)) break;
+                    KSA_BT_WAIT_END(bt_wait_c); }
+                    { KSA_BT_WAIT_BEGIN();
+                    bt_product(tX, sm.a1(), sm.b1(s1));
+                    tc_commit(sm.bar(BB_XFULL));
+                    KSA_BT_WAIT_END(bt_iss_x); }
+                }
+                // P^T and dS^T stand in Y's columns (row warp 0 checked the stage of Y_{j+1} before it arrived)
                 { KSA_BT_WAIT_BEGIN();
                   if (!bt_wait(sm.bar(BB_PB), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                   KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
+                KSA_BT_WAIT_BEGIN();
+                bt_accumulate(tDV, tY + 16, sm.b2(j & 1), j == 0);                          // dV += P^T dO_j
+                tc_commit(sm.bar(BB_B2EMPTY + (j & 1)));                                    // ... then its dO stage is free
                 bt_accumulate(tDK, tY, sm.b1(j % kB1Stages), j == 0);                       // dK += dS^T Q_j
+                tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // ... then its Q stage is free
                 if (j + 1 < J) { bt_product(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
+                KSA_BT_WAIT_END(bt_iss_acc);
             }
             tc_commit(sm.bar(BB_OFULL));
 #if defined(KSA_BWD_TRACE) && KSA_BWD_TRACE == 4
             if (summ && blockIdx.x == 1 && blockIdx.y == 4 && blockIdx.z == 0) {
                 g_btrace[0][0] = make_uint2(bt_wait_a, bt_wait_b);
                 g_btrace[0][1] = make_uint2((uint32_t)clock() - bt_loop0, (uint32_t)J);
-                g_btrace_cnt[0] = 2;
+                g_btrace[0][2] = make_uint2(bt_wait_c, bt_iss_x);
+                g_btrace[0][3] = make_uint2(bt_iss_acc, 0u);
+                g_btrace_cnt[0] = 4;
             }
 #endif
         }
@@ -377,17 +394,15 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         int qt = seg0, g = 0;
         int iq0 = (seg0 * 128 + 32 * cg) / a.k, ir0 = (seg0 * 128 + 32 * cg) - iq0 * a.k;
         for (int j = 0; j < J && alive; ++j) {
-            if (scalar_writer && j + 1 < J) fetch(g + 1 == G ? qt + 1 : qt, g + 1 == G ? 0 : g + 1);   // lands while this tile is worked on
+            if (j + 1 < J) fetch(g + 1 == G ? qt + 1 : qt, g + 1 == G ? 0 : g + 1);   // lands while this tile is worked on
             const float* lse_c = rows + (j & 1) * 256 + 32 * cg;          // this warp's 32 columns
             const float* dl_c = lse_c + 128;
             const int i0 = qt * 128 + 32 * cg;                            // first query of the block
             const int iq1 = iq0 + q31 + (ir0 + r31 >= a.k ? 1 : 0);       // chunk of the block's last query
-            // ---------------- phase A: P^T = exp2(S^T scale - lse) ----------------
+            // ---------------- phase A: P^T = exp2(S^T scale - lse), kept in registers ----------------
             if (!bt_wait_warp(sm.bar(BB_XFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
             KSA_BT(bt_role, 10);
             tc_fence_after();
-            // X_j was issued after dV += P^T dO_{j-1}: that tile's dO stage is free
-            if (warp == 0 && lane == 0 && j >= 1) mbar_arrive(sm.bar(BB_B2EMPTY + ((j - 1) & 1)));
             // all pairs of the block visible / none (rows past the streams drop out by themselves: zero K / V
             // rows are discarded at the end, padding queries have lse = +inf)
             bool full, none;
@@ -406,7 +421,13 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                 tmem_ld16(tXc, x0);
                 tmem_ld16(tXc + 16, x1);
                 tc_wait_ld();
-                KSA_BT(bt_role, 11);
+            }
+            // X_j is in registers: the issuer may start X_{j+1} while the exponentials run
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.bar(BB_PA));
+            KSA_BT(bt_role, 11);
+            if (!none) {
                 if (full) {
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
@@ -425,41 +446,24 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     }
                 }
             }
-            {
-                uint32_t pp[16];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    pp[c] = pack_bf16x2(__uint_as_float(x0[2 * c]), __uint_as_float(x0[2 * c + 1]));
-                    pp[8 + c] = pack_bf16x2(__uint_as_float(x1[2 * c]), __uint_as_float(x1[2 * c + 1]));
-                }
-                tmem_st16(tXc, pp);                                       // over the block's own first 16 columns
-                // X_j was complete, so every warp is past phase A of tile j - 1: its lse buffer may be overwritten
-                // (the arrival below publishes the values: X_{j+1} is only issued after it)
-                if (scalar_writer && j + 1 < J) rows[((j + 1) & 1) * 256 + 32 * cg + lane] = n_lse;
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    if (warp == 0 && j + 1 < J)                            // warp 0 vouches for the stage of X_{j+1}
-                        bt_wait(sm.bar(BB_B1FULL + (j + 1) % kB1Stages), ((j + 1) / kB1Stages) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
-                    mbar_arrive(sm.bar(BB_PA));
-                }
-            }
             KSA_BT(bt_role, 12);
-            // ---------------- phase B: dS^T = P^T (dP^T - delta) ----------------
+            // ---------------- phase B: dS^T = P^T (dP^T - delta); both as bf16 over Y's own columns ----------------
             if (!bt_wait_warp(sm.bar(BB_YFULL), j & 1, sm.abort_addr(), a.status, kStatusWaitSFull, lane)) { alive = false; break; }
             KSA_BT(bt_role, 13);
             tc_fence_after();
-            // Y_j was issued after dK += dS^T Q_{j-1}: that tile's Q stage is free
-            if (warp == 0 && lane == 0 && j >= 1) mbar_arrive(sm.bar(BB_B1EMPTY + (j - 1) % kB1Stages));
+            // Y_j was issued after every warp's arrival for tile j - 1: that tile's scalars may be overwritten
+            if (j + 1 < J) {
+                rows[((j + 1) & 1) * 256 + 32 * cg + lane] = n_lse;
+                rows[((j + 1) & 1) * 256 + 128 + 32 * cg + lane] = n_dl;
+            }
             {
-                uint32_t dd[16];
+                uint32_t dd[16], pp[16];                                  // dS^T: columns 0 .. 15 of the block, P^T: 16 .. 31
                 if (none) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) dd[c] = 0u;
+                    for (int c = 0; c < 16; ++c) dd[c] = pp[c] = 0u;
                 } else {
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
+                    for (int half = 1; half >= 0; --half) {
                         uint32_t ys[16];
                         tmem_ld16(tYc + half * 16, ys);
                         tc_wait_ld();
@@ -468,12 +472,12 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                             const float p0 = __uint_as_float(half ? x1[c] : x0[c]), p1 = __uint_as_float(half ? x1[c + 1] : x0[c + 1]);
                             dd[half * 8 + (c >> 1)] = pack_bf16x2(p0 * (__uint_as_float(ys[c]) - dl_c[half * 16 + c]),
                                                                   p1 * (__uint_as_float(ys[c + 1]) - dl_c[half * 16 + c + 1]));
+                            pp[half * 8 + (c >> 1)] = pack_bf16x2(p0, p1);
                         }
                     }
                 }
-                tmem_st16(tYc, dd);
-                // Y_j was complete, so every warp is past phase B of tile j - 1: its delta buffer may be overwritten
-                if (scalar_writer && j + 1 < J) rows[((j + 1) & 1) * 256 + 128 + 32 * cg + lane] = n_dl;
+                tmem_st16(tYc, dd);                                       // all 32 columns of dP^T have been read
+                tmem_st16(tYc + 16, pp);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
