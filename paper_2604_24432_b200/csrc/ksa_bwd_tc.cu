@@ -11,10 +11,13 @@
 //   dK / dV  key-stationary and transposed: A1 = K tile, A2 = V tile (text or summary stream), B1 = Q tile,
 //            B2 = dO tile of the (query tile, query head) pairs that see the keys; X = S^T, Y = dP^T.
 //            The warps hand X back as soon as it is in their registers, so X_{j+1} runs beside the
-//            exponentials of tile j; phase B writes dS^T over columns 0 .. 15 and P^T over columns 16 .. 31 of
-//            each warp's 32-column block of Y.  Pipe order per j: X_{j+1}, dV += P^T dO_j, dK += dS^T Q_j,
-//            Y_{j+1}.  At the end each key row adds dV and scale * dK to the fp32 accumulators of its stream
-//            (vector atomics: several segments and the summary-row kernel add to the same rows).
+//            exponentials of tile j; phase B goes through each warp's 32-column block of Y in two halves of
+//            16 queries and writes dS^T over the first 8 and P^T over the other 8 columns of the half just
+//            read, with one arrival per half: the accumulations over the first halves (k-steps 0, 2, 4, 6)
+//            run beside the arithmetic of the second.  Pipe order per j: X_{j+1}, dV += P^T dO_j and
+//            dK += dS^T Q_j (even k-steps, then odd), Y_{j+1}.  At the end each key row adds dV and
+//            scale * dK to the fp32 accumulators of its stream (vector atomics: several segments and the
+//            summary-row kernel add to the same rows).
 //   dQ       query-stationary: A1 = Q tile, A2 = dO tile, B1 = K tile, B2 = V tile over the visible
 //            summary tiles, then the visible text tiles (Eq. 3); X = S, Y = dP.  One accumulator leaves
 //            room for a second Y buffer (columns from 384), so both products of tile j + 1 are issued
@@ -191,6 +194,18 @@ __device__ __forceinline__ void bt_accumulate(uint32_t tmem_d, uint32_t tmem_a, 
         mma_ts(tmem_d, tmem_a + (kk >> 1) * 32 + (kk & 1) * 8, bd + (uint32_t)((kk * 2048) >> 4), idesc, (!first || kk > 0) ? 1u : 0u);
 }
 
+// Half of such an accumulation for the dK / dV kernel, whose row warps hand their 32-column blocks over in two
+// halves of 16 query columns: the four k-steps 2 c + odd, whose 16 x bf16 operand stands in the 8 columns at
+// tmem_a + 32 c + 16 odd (tmem_a already points at dS^T, or 8 columns further at P^T).
+__device__ __forceinline__ void bt_accumulate_half(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_tile, int odd, bool first)
+{
+    constexpr uint32_t idesc = make_idesc_bf16(128, 128, true);
+    const uint64_t bd = make_smem_desc_sw128(b_tile, 16384, 1024);
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        mma_ts(tmem_d, tmem_a + c * 32 + odd * 16, bd + (uint32_t)(((2 * c + odd) * 2048) >> 4), idesc, (!first || c > 0) ? 1u : 0u);
+}
+
 // ---- producer helpers (one thread) ----------------------------------------------------------------
 // The two 64-column halves of a 128-row tile.  Packed streams: rows pos .. pos + 127 of a 3-D map.  Direct mode
 // (no packed copies: every sequence a whole number of chunks): chunks pos .. of a 4-D view [D, rows per chunk,
@@ -349,15 +364,20 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     tc_commit(sm.bar(BB_XFULL));
                     KSA_BT_WAIT_END(bt_iss_x); }
                 }
-                // P^T and dS^T stand in Y's columns (row warp 0 checked the stage of Y_{j+1} before it arrived)
+                // dS^T and P^T of the first 16 queries of every block stand in Y's columns: the even k-steps
                 { KSA_BT_WAIT_BEGIN();
                   if (!bt_wait(sm.bar(BB_PB), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                   KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
                 KSA_BT_WAIT_BEGIN();
-                bt_accumulate(tDV, tY + 16, sm.b2(j & 1), j == 0);                          // dV += P^T dO_j
+                bt_accumulate_half(tDV, tY + 8, sm.b2(j & 1), 0, j == 0);                   // dV += P^T dO_j
+                bt_accumulate_half(tDK, tY, sm.b1(j % kB1Stages), 0, j == 0);               // dK += dS^T Q_j
+                // ... the other 16 (row warp 0 checked the stage of Y_{j+1} before it arrived): the odd k-steps
+                if (!bt_wait(sm.bar(BB_PB2), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
+                tc_fence_after();
+                bt_accumulate_half(tDV, tY + 8, sm.b2(j & 1), 1, false);
                 tc_commit(sm.bar(BB_B2EMPTY + (j & 1)));                                    // ... then its dO stage is free
-                bt_accumulate(tDK, tY, sm.b1(j % kB1Stages), j == 0);                       // dK += dS^T Q_j
+                bt_accumulate_half(tDK, tY, sm.b1(j % kB1Stages), 1, false);
                 tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // ... then its Q stage is free
                 if (j + 1 < J) { bt_product(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
                 KSA_BT_WAIT_END(bt_iss_acc);
@@ -456,35 +476,34 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                 rows[((j + 1) & 1) * 256 + 32 * cg + lane] = n_lse;
                 rows[((j + 1) & 1) * 256 + 128 + 32 * cg + lane] = n_dl;
             }
-            {
-                uint32_t dd[16], pp[16];                                  // dS^T: columns 0 .. 15 of the block, P^T: 16 .. 31
+            // handed over in two halves of 16 queries, so that the accumulations of the first run beside the
+            // arithmetic of the second: columns 16 half + 0 .. 7 take dS^T, 16 half + 8 .. 15 take P^T
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t o[16];
                 if (none) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) dd[c] = pp[c] = 0u;
+                    for (int c = 0; c < 16; ++c) o[c] = 0u;
                 } else {
+                    uint32_t ys[16];
+                    tmem_ld16(tYc + half * 16, ys);
+                    tc_wait_ld();
 #pragma unroll
-                    for (int half = 1; half >= 0; --half) {
-                        uint32_t ys[16];
-                        tmem_ld16(tYc + half * 16, ys);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 16; c += 2) {
-                            const float p0 = __uint_as_float(half ? x1[c] : x0[c]), p1 = __uint_as_float(half ? x1[c + 1] : x0[c + 1]);
-                            dd[half * 8 + (c >> 1)] = pack_bf16x2(p0 * (__uint_as_float(ys[c]) - dl_c[half * 16 + c]),
-                                                                  p1 * (__uint_as_float(ys[c + 1]) - dl_c[half * 16 + c + 1]));
-                            pp[half * 8 + (c >> 1)] = pack_bf16x2(p0, p1);
-                        }
+                    for (int c = 0; c < 16; c += 2) {
+                        const float p0 = __uint_as_float(half ? x1[c] : x0[c]), p1 = __uint_as_float(half ? x1[c + 1] : x0[c + 1]);
+                        o[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(ys[c]) - dl_c[half * 16 + c]),
+                                                p1 * (__uint_as_float(ys[c + 1]) - dl_c[half * 16 + c + 1]));
+                        o[8 + (c >> 1)] = pack_bf16x2(p0, p1);
                     }
                 }
-                tmem_st16(tYc, dd);                                       // all 32 columns of dP^T have been read
-                tmem_st16(tYc + 16, pp);
+                tmem_st16(tYc + half * 16, o);                            // over the 16 columns of dP^T just read
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    if (warp == 0 && j + 1 < J)                            // warp 0 vouches for the stage of Y_{j+1}
+                    if (half == 1 && warp == 0 && j + 1 < J)               // warp 0 vouches for the stage of Y_{j+1}
                         bt_wait(sm.bar(BB_B2FULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, sm.abort_addr(), a.status, kStatusWaitQFull);
-                    mbar_arrive(sm.bar(BB_PB));
+                    mbar_arrive(sm.bar(half ? BB_PB2 : BB_PB));
                 }
             }
             KSA_BT(bt_role, 14);
