@@ -151,83 +151,73 @@ __global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
 }
 
 // Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row).
-// A block stages the K and V rows of kSummChunks consecutive chunks of one KV head in shared
-// memory (each row is read from global memory once, whatever the GQA group size), then its
-// warps take the (summary row, query head) tasks of those chunks: every key of the row is read
-// from shared memory before any is used, and the per-key dot products are reduced across the
-// warp together (independent shuffle chains).
+// One warp per (chunk, KV head).  Its lanes form four groups of eight: a group takes one (summary row, query
+// head) task at a time, each lane D / 8 consecutive elements of the head dimension (16-byte vectors), so a dot
+// product needs three shuffle steps instead of five and the four groups read the very same K / V addresses
+// (one transaction per warp: every K / V row is fetched once per pass over four tasks, from L1 after the
+// first).  No shared memory, no block-wide barrier; all loads of a pass are independent of its arithmetic.
 constexpr int kSummMaxKeys = 12;
-constexpr int kSummChunks = 8;
+constexpr int kSummChunks = 8;      // chunks (= warps) per block
 
 template <int D>
 __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 {
-    constexpr int E = D / 32;                     // dimensions per lane: 4 (8 bytes) or 2 (4 bytes)
-    using Vec = typename std::conditional<E == 4, uint2, uint32_t>::type;
-    __shared__ __align__(16) uint16_t sK[kSummChunks * kSummMaxKeys * D];
-    __shared__ __align__(16) uint16_t sV[kSummChunks * kSummMaxKeys * D];
+    constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
+    constexpr int V4 = E / 8;
     const bool ranged = a.r_seq >= 0;
     const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const int hk = blockIdx.z;
     // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
     const int j_first = ranged ? a.r_summ0 / a.m : 0;
     const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
-    const int j0 = j_first + blockIdx.x * kSummChunks;
-    if (j0 >= j_end) return;
-    const int nch = min(kSummChunks, j_end - j0);
+    const int j = j_first + blockIdx.x * kSummChunks + (threadIdx.x >> 5);
+    if (j >= j_end) return;                                            // warp-uniform
+    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
     const int s = a.k + a.m;
     const int G = a.Hq / a.Hkv;
-    const int64_t row0 = sq.aug_off + (int64_t)j0 * s;
-    // stage nch * s rows of K and V (16-byte vectors)
-    {
-        const int vecs = D / 8;
-        const int total = nch * s * vecs;
-        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
-            const int rr = idx / vecs, vv = idx - rr * vecs;
-            const uint4 kx = *reinterpret_cast<const uint4*>(a.kx + (row0 + rr) * a.k_st + (int64_t)hk * a.k_sh + vv * 8);
-            const uint4 vx = *reinterpret_cast<const uint4*>(a.v + (row0 + rr) * a.v_st + (int64_t)hk * a.v_sh + vv * 8);
-            *reinterpret_cast<uint4*>(sK + rr * D + vv * 8) = kx;
-            *reinterpret_cast<uint4*>(sV + rr * D + vv * 8) = vx;
-        }
-    }
-    __syncthreads();
-    const int lane = threadIdx.x & 31;
-    const int wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    auto unpack = [](const Vec& raw, float (&f)[E]) {
-        const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw);
+    const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
+    const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
+    const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
+    auto unpack = [](const uint4& raw, float* f) {
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-        for (int e = 0; e < E; e += 2) {
-            f[e] = __uint_as_float(w[e / 2] << 16);
-            f[e + 1] = __uint_as_float(w[e / 2] & 0xffff0000u);
+        for (int e = 0; e < 4; ++e) {
+            f[2 * e] = __uint_as_float(w[e] << 16);
+            f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
         }
     };
-    const int tasks = nch * a.m * G;
-    for (int task = wid; task < tasks; task += nwarps) {
-        const int g = task % G;
-        const int cr = task / G;
-        const int c = cr / a.m, r = cr - c * a.m;
+    const int tasks = a.m * G;
+    for (int t0 = 0; t0 < tasks; t0 += 4) {
+        const int task = t0 + grp;
+        const bool live = task < tasks;
+        const int tk = live ? task : tasks - 1;                        // idle groups shadow the last task (no stores)
+        const int r = tk / G, g = tk - r * G;
         const int h = hk * G + g;
-        const int64_t qrow = row0 + (int64_t)c * s + a.k + r;
-        const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));     // own-chunk text (+ own summaries 0..r)
-        const Vec qraw = *reinterpret_cast<const Vec*>(a.q + qrow * a.q_st + (int64_t)h * a.q_sh + lane * E);
-        const uint16_t* kbase = sK + c * s * D + lane * E;
-        const uint16_t* vbase = sV + c * s * D + lane * E;
+        const int64_t qrow = row0 + a.k + r;
+        const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));           // own-chunk text (+ own summaries 0..r)
         float qv[E];
-        unpack(qraw, qv);
+        {
+            const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + sub * E;
+#pragma unroll
+            for (int c = 0; c < V4; ++c) unpack(*reinterpret_cast<const uint4*>(qp + 8 * c), qv + 8 * c);
+        }
         float x[kSummMaxKeys];
 #pragma unroll
         for (int t = 0; t < kSummMaxKeys; ++t) {
             float dot = 0.f;
-            if (t < nk) {
-                float kf[E];
-                unpack(*reinterpret_cast<const Vec*>(kbase + t * D), kf);
+            if (t < s) {                                               // uniform: rows of the chunk
 #pragma unroll
-                for (int e = 0; e < E; ++e) dot = fmaf(qv[e], kf[e], dot);
+                for (int c = 0; c < V4; ++c) {
+                    float kf[8];
+                    unpack(*reinterpret_cast<const uint4*>(kp + (int64_t)t * a.k_st + 8 * c), kf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) dot = fmaf(qv[8 * c + e], kf[e], dot);
+                }
             }
             x[t] = dot;
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
+        for (int o = 4; o > 0; o >>= 1) {
 #pragma unroll
             for (int t = 0; t < kSummMaxKeys; ++t)
                 if (t < s) x[t] += __shfl_xor_sync(0xffffffffu, x[t], o);
@@ -243,24 +233,32 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
 #pragma unroll
         for (int t = 0; t < kSummMaxKeys; ++t) {
-            if (t < nk) {
-                const float p = __expf(x[t] - mx);
+            if (t < s) {
+                const float p = (t < nk) ? __expf(x[t] - mx) : 0.f;
                 l += p;
-                float vf[E];
-                unpack(*reinterpret_cast<const Vec*>(vbase + t * D), vf);
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
+                for (int c = 0; c < V4; ++c) {
+                    float vf[8];
+                    unpack(*reinterpret_cast<const uint4*>(vp + (int64_t)t * a.v_st + 8 * c), vf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[8 * c + e] = fmaf(p, vf[e], acc[8 * c + e]);
+                }
             }
         }
-        const float inv = 1.f / l;
-        uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + lane * E;
-        Vec ov;
-        uint32_t* ow = reinterpret_cast<uint32_t*>(&ov);
+        if (live) {
+            const float inv = 1.f / l;
+            uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * E;
 #pragma unroll
-        for (int e = 0; e < E; e += 2)
-            ow[e / 2] = (uint32_t)float_to_bf16_bits(acc[e] * inv) | ((uint32_t)float_to_bf16_bits(acc[e + 1] * inv) << 16);
-        *reinterpret_cast<Vec*>(op) = ov;
-        if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
+            for (int c = 0; c < V4; ++c) {
+                uint4 ov;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&ov);
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    ow[e] = (uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e] * inv) | ((uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e + 1] * inv) << 16);
+                *reinterpret_cast<uint4*>(op + 8 * c) = ov;
+            }
+            if (sub == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
+        }
     }
 }
 
