@@ -95,59 +95,135 @@ cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream)
 }
 
 // ---------------------------------------------------------------------------------------
-// Summary rows (Sec. 2.2.1, first bullet).  One warp per (summary row, query head): the
-// keys are the contiguous augmented rows j*(k+m) .. j*(k+m) + k - 1 (+ r + 1 own-chunk
-// summaries unless KSA_FLAG_SUMMARY_TEXT_ONLY).  Each lane owns D/32 dimensions.
+// Summary rows (Sec. 2.2.1, first bullet), chunks of any length.  The keys of summary r of chunk j are the
+// contiguous augmented rows j*(k+m) .. j*(k+m) + k - 1 (+ r + 1 own-chunk summaries unless
+// KSA_FLAG_SUMMARY_TEXT_ONLY).  One warp per (chunk, KV head, block of eight (summary row, query head) tasks),
+// the task blocks of a chunk in neighbouring warps;
+// its lanes form four groups of eight, a group takes one task at a time and each lane D / 8 consecutive
+// elements of the head dimension (16-byte vectors; three shuffle steps per dot product; the four groups read
+// the same K / V addresses).  The keys go by in batches of kSummBatch with a running maximum and sum.
 // ---------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
+constexpr int kSummBatch = 8;
+constexpr int kSummTaskBlock = 8;   // tasks per warp
+constexpr int kSummChunks = 8;      // short chunks: chunks (= warps) per block
+
+__device__ __forceinline__ void summ_unpack(const uint4& raw, float* f)
 {
-    constexpr int E = D / 32;
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        f[2 * e] = __uint_as_float(w[e] << 16);
+        f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(256, 3) ksa_summary_kernel(KernelArgs a)
+{
+    constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
+    constexpr int V4 = E / 8;
     const bool ranged = a.r_seq >= 0;
     const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int u_first = ranged ? a.r_summ0 : 0;
-    const int64_t total = (int64_t)((ranged ? a.r_summq1 : sq.n_summ) - u_first) * a.Hq;
-    if (warp >= total) return;
-    const int u = u_first + (int)(warp / a.Hq);
-    const int h = (int)(warp % a.Hq);
-    const int hk = h / (a.Hq / a.Hkv);
-    const int j = u / a.m, r = u - j * a.m;
+    const int hk = blockIdx.z;
+    const int G = a.Hq / a.Hkv;
+    const int tasks = a.m * G;
+    const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;
+    // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
+    const int j_first = ranged ? a.r_summ0 / a.m : 0;
+    const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
+    // consecutive warps take the task blocks of one chunk (they read the same K / V rows), then the next chunk's
+    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int j = j_first + (int)(gw / task_blocks);
+    if (j >= j_end) return;                                            // warp-uniform
+    const int task_lo = (int)(gw % task_blocks) * kSummTaskBlock;
+    const int task_hi = min(tasks, task_lo + kSummTaskBlock);
+    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
     const int s = a.k + a.m;
-    const int64_t key0 = sq.aug_off + (int64_t)j * s;
-    const int64_t qrow = key0 + a.k + r;
-    const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));
-
-    float qv[E], acc[E];
-    {
-        const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + lane * E;
+    const int own = (a.flags & 1u) ? 0 : 1;                            // a summary sees the chunk's summaries up to itself
+    const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
+    const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
+    const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
+    for (int t0 = task_lo; t0 < task_hi; t0 += 4) {
+        const int task = t0 + grp;
+        const bool live = task < task_hi;
+        const int tk = live ? task : task_hi - 1;                      // idle groups shadow the last task (no stores)
+        const int r = tk / G, g = tk - r * G;
+        const int h = hk * G + g;
+        const int64_t qrow = row0 + a.k + r;
+        const int nk = a.k + own * (r + 1);
+        const int nk_max = a.k + own * ((min(t0 + 3, task_hi - 1)) / G + 1);   // of the four tasks: uniform over the warp
+        float qv[E], acc[E];
+        {
+            const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + sub * E;
 #pragma unroll
-        for (int e = 0; e < E; ++e) { qv[e] = bf16_bits_to_float(qp[e]); acc[e] = 0.f; }
+            for (int c = 0; c < V4; ++c) summ_unpack(*reinterpret_cast<const uint4*>(qp + 8 * c), qv + 8 * c);
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        float mx = -INFINITY, l = 0.f;
+        for (int b0 = 0; b0 < nk_max; b0 += kSummBatch) {
+            float x[kSummBatch];
+#pragma unroll
+            for (int i = 0; i < kSummBatch; ++i) {
+                float dot = 0.f;
+                if (b0 + i < nk_max) {
+#pragma unroll
+                    for (int c = 0; c < V4; ++c) {
+                        float kf[8];
+                        summ_unpack(*reinterpret_cast<const uint4*>(kp + (int64_t)(b0 + i) * a.k_st + 8 * c), kf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) dot = fmaf(qv[8 * c + e], kf[e], dot);
+                    }
+                }
+                x[i] = dot;
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+#pragma unroll
+                for (int i = 0; i < kSummBatch; ++i) x[i] += __shfl_xor_sync(0xffffffffu, x[i], o);
+            }
+            float mn = mx;
+#pragma unroll
+            for (int i = 0; i < kSummBatch; ++i) {
+                x[i] = (b0 + i < nk) ? x[i] * a.scale : -INFINITY;
+                mn = fmaxf(mn, x[i]);
+            }
+            // key 0 is visible to every task, so mn is finite from the first batch on
+            const float alpha = __expf(mx - mn);                       // exp(-inf) = 0 on the first batch
+            mx = mn;
+            l *= alpha;
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] *= alpha;
+#pragma unroll
+            for (int i = 0; i < kSummBatch; ++i) {
+                if (b0 + i < nk_max) {
+                    const float p = __expf(x[i] - mn);                 // 0 on the keys this task does not see
+                    l += p;
+#pragma unroll
+                    for (int c = 0; c < V4; ++c) {
+                        float vf[8];
+                        summ_unpack(*reinterpret_cast<const uint4*>(vp + (int64_t)(b0 + i) * a.v_st + 8 * c), vf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[8 * c + e] = fmaf(p, vf[e], acc[8 * c + e]);
+                    }
+                }
+            }
+        }
+        if (live) {
+            const float inv = 1.f / l;
+            uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * E;
+#pragma unroll
+            for (int c = 0; c < V4; ++c) {
+                uint4 ov;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&ov);
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    ow[e] = (uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e] * inv) | ((uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e + 1] * inv) << 16);
+                *reinterpret_cast<uint4*>(op + 8 * c) = ov;
+            }
+            if (sub == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
+        }
     }
-    float mx = -INFINITY, l = 0.f;
-    for (int t = 0; t < nk; ++t) {
-        const uint16_t* kp = a.kx + (key0 + t) * a.k_st + (int64_t)hk * a.k_sh + lane * E;
-        float dot = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) dot = fmaf(qv[e], bf16_bits_to_float(kp[e]), dot);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        const float x = dot * a.scale;
-        const float mn = fmaxf(mx, x);
-        const float alpha = __expf(mx - mn);     // exp(-inf) = 0 on the first key
-        const float p = __expf(x - mn);
-        l = l * alpha + p;
-        const uint16_t* vp = a.v + (key0 + t) * a.v_st + (int64_t)hk * a.v_sh + lane * E;
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] = fmaf(acc[e], alpha, p * bf16_bits_to_float(vp[e]));
-        mx = mn;
-    }
-    const float inv = 1.f / l;
-    uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
-    if (lane == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
 }
 
 // Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row).
@@ -157,7 +233,6 @@ __global__ void __launch_bounds__(256) ksa_summary_kernel(KernelArgs a)
 // (one transaction per warp: every K / V row is fetched once per pass over four tasks, from L1 after the
 // first).  No shared memory, no block-wide barrier; all loads of a pass are independent of its arithmetic.
 constexpr int kSummMaxKeys = 12;
-constexpr int kSummChunks = 8;      // chunks (= warps) per block
 
 template <int D>
 __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
@@ -269,18 +344,18 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
     const int rows = a.r_seq >= 0 ? (a.r_summq1 - a.r_summ0) : a.max_n_summ;
     if (rows <= 0) return cudaSuccess;
     const unsigned ny = a.r_seq >= 0 ? 1u : (unsigned)a.num_seqs;
-    const int64_t warps = (int64_t)rows * a.Hq;
-    int64_t blocks = (warps + 7) / 8;
-    if (blocks < 1) blocks = 1;
-    dim3 grid((unsigned)blocks, ny, 1);
+    const int max_chunks = rows / a.m;
+    const int chunk_groups = (max_chunks + kSummChunks - 1) / kSummChunks;
     if (a.k + a.m <= kSummMaxKeys) {
-        const int max_chunks = rows / a.m;
-        dim3 g2((unsigned)((max_chunks + kSummChunks - 1) / kSummChunks), ny, (unsigned)a.Hkv);
+        dim3 g2((unsigned)chunk_groups, ny, (unsigned)a.Hkv);
         if (a.D == 128) ksa_summary_short_kernel<128><<<g2, 256, 0, stream>>>(a);
         else            ksa_summary_short_kernel<64><<<g2, 256, 0, stream>>>(a);
     } else {
-        if (a.D == 128) ksa_summary_kernel<128><<<grid, 256, 0, stream>>>(a);
-        else            ksa_summary_kernel<64><<<grid, 256, 0, stream>>>(a);
+        const int tasks = a.m * (a.Hq / a.Hkv);
+        const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;
+        dim3 g3((unsigned)(((int64_t)max_chunks * task_blocks + 7) / 8), ny, (unsigned)a.Hkv);
+        if (a.D == 128) ksa_summary_kernel<128><<<g3, 256, 0, stream>>>(a);
+        else            ksa_summary_kernel<64><<<g3, 256, 0, stream>>>(a);
     }
     return cudaGetLastError();
 }
