@@ -107,6 +107,18 @@ constexpr int kSummBatch = 8;
 constexpr int kSummTaskBlock = 8;   // tasks per warp
 constexpr int kSummChunks = 8;      // short chunks: chunks (= warps) per block
 
+// The warp asks for the 128-byte lines of rows [0, rows) of one head (D elements per row, row stride st elements)
+// ahead of their use: the loads that follow then find them in L1 instead of waiting for L2 / HBM one key at a time.
+template <int D>
+__device__ __forceinline__ void summ_prefetch_rows(const uint16_t* base, int64_t st, int rows, int lane)
+{
+    constexpr int kLines = D * 2 / 128 > 0 ? D * 2 / 128 : 1;
+    for (int idx = lane; idx < rows * kLines; idx += 32) {
+        const uint16_t* p = base + (int64_t)(idx / kLines) * st + (idx % kLines) * 64;
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+    }
+}
+
 __device__ __forceinline__ void summ_unpack(const uint4& raw, float* f)
 {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -118,7 +130,7 @@ __device__ __forceinline__ void summ_unpack(const uint4& raw, float* f)
 }
 
 template <int D>
-__global__ void __launch_bounds__(256, 3) ksa_summary_kernel(KernelArgs a)
+__global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
 {
     constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
     constexpr int V4 = E / 8;
@@ -143,6 +155,11 @@ __global__ void __launch_bounds__(256, 3) ksa_summary_kernel(KernelArgs a)
     const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
     const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
     const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
+    {
+        const int rows_seen = a.k + own * ((task_hi - 1) / G + 1);     // keys of the warp's last task
+        summ_prefetch_rows<D>(a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh, a.k_st, rows_seen, lane);
+        summ_prefetch_rows<D>(a.v + row0 * a.v_st + (int64_t)hk * a.v_sh, a.v_st, rows_seen, lane);
+    }
     for (int t0 = task_lo; t0 < task_hi; t0 += 4) {
         const int task = t0 + grp;
         const bool live = task < task_hi;
@@ -253,6 +270,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
     const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
     const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
     const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
+    summ_prefetch_rows<D>(a.v + row0 * a.v_st + (int64_t)hk * a.v_sh, a.v_st, s, lane);    // V is used last: ask for it first
     auto unpack = [](const uint4& raw, float* f) {
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
