@@ -244,11 +244,12 @@ __global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
 }
 
 // Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row).
-// One warp per (chunk, KV head).  Its lanes form four groups of eight: a group takes one (summary row, query
-// head) task at a time, each lane D / 8 consecutive elements of the head dimension (16-byte vectors), so a dot
-// product needs three shuffle steps instead of five and the four groups read the very same K / V addresses
-// (one transaction per warp: every K / V row is fetched once per pass over four tasks, from L1 after the
-// first).  No shared memory, no block-wide barrier; all loads of a pass are independent of its arithmetic.
+// A block stages the K and V rows of kSummChunks consecutive chunks of one KV head in shared memory (each row
+// is read from global memory once, whatever the GQA group size, with every load of the block in flight at
+// once); then one warp per chunk: its lanes form four groups of eight, a group takes one (summary row, query
+// head) task at a time, each lane 8 consecutive elements of each 64-element half of the head dimension
+// (16-byte vectors, neighbouring lanes on neighbouring banks), so a dot product needs three shuffle steps
+// and the four groups read the very same shared-memory addresses.
 constexpr int kSummMaxKeys = 12;
 
 template <int D>
@@ -256,21 +257,41 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 {
     constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
     constexpr int V4 = E / 8;
+    __shared__ __align__(16) uint16_t sK[kSummChunks * kSummMaxKeys * D];
+    __shared__ __align__(16) uint16_t sV[kSummChunks * kSummMaxKeys * D];
     const bool ranged = a.r_seq >= 0;
     const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const int hk = blockIdx.z;
     // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
     const int j_first = ranged ? a.r_summ0 / a.m : 0;
     const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
-    const int j = j_first + blockIdx.x * kSummChunks + (threadIdx.x >> 5);
-    if (j >= j_end) return;                                            // warp-uniform
-    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
+    const int j0 = j_first + blockIdx.x * kSummChunks;
+    if (j0 >= j_end) return;                                           // block-uniform
+    const int nch = min(kSummChunks, j_end - j0);
     const int s = a.k + a.m;
     const int G = a.Hq / a.Hkv;
+    // the block's nch * s rows of K and V of this KV head (contiguous augmented rows), 16-byte vectors
+    {
+        constexpr int vecs = D / 8;
+        const int64_t r0 = sq.aug_off + (int64_t)j0 * s;
+        const int total = nch * s * vecs;
+        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+            const int rr = idx / vecs, vv = idx - rr * vecs;
+            const uint4 kx = *reinterpret_cast<const uint4*>(a.kx + (r0 + rr) * a.k_st + (int64_t)hk * a.k_sh + vv * 8);
+            const uint4 vx = *reinterpret_cast<const uint4*>(a.v + (r0 + rr) * a.v_st + (int64_t)hk * a.v_sh + vv * 8);
+            *reinterpret_cast<uint4*>(sK + rr * D + vv * 8) = kx;
+            *reinterpret_cast<uint4*>(sV + rr * D + vv * 8) = vx;
+        }
+    }
+    __syncthreads();
+    const int wid = threadIdx.x >> 5;
+    if (wid >= nch) return;                                            // warp-uniform, after the only barrier
+    const int j = j0 + wid;
+    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
     const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
-    const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
-    const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
-    summ_prefetch_rows<D>(a.v + row0 * a.v_st + (int64_t)hk * a.v_sh, a.v_st, s, lane);    // V is used last: ask for it first
+    // a lane's elements: 8 sub .. 8 sub + 7 of each 64-element half (neighbouring lanes read neighbouring 16 bytes)
+    const uint16_t* kp = sK + wid * s * D + sub * 8;
+    const uint16_t* vp = sV + wid * s * D + sub * 8;
     auto unpack = [](const uint4& raw, float* f) {
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -290,9 +311,9 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
         const int nk = a.k + ((a.flags & 1u) ? 0 : (r + 1));           // own-chunk text (+ own summaries 0..r)
         float qv[E];
         {
-            const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + sub * E;
+            const uint16_t* qp = a.q + qrow * a.q_st + (int64_t)h * a.q_sh + sub * 8;
 #pragma unroll
-            for (int c = 0; c < V4; ++c) unpack(*reinterpret_cast<const uint4*>(qp + 8 * c), qv + 8 * c);
+            for (int c = 0; c < V4; ++c) unpack(*reinterpret_cast<const uint4*>(qp + 64 * c), qv + 8 * c);
         }
         float x[kSummMaxKeys];
 #pragma unroll
@@ -302,7 +323,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 #pragma unroll
                 for (int c = 0; c < V4; ++c) {
                     float kf[8];
-                    unpack(*reinterpret_cast<const uint4*>(kp + (int64_t)t * a.k_st + 8 * c), kf);
+                    unpack(*reinterpret_cast<const uint4*>(kp + t * D + 64 * c), kf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) dot = fmaf(qv[8 * c + e], kf[e], dot);
                 }
@@ -332,7 +353,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 #pragma unroll
                 for (int c = 0; c < V4; ++c) {
                     float vf[8];
-                    unpack(*reinterpret_cast<const uint4*>(vp + (int64_t)t * a.v_st + 8 * c), vf);
+                    unpack(*reinterpret_cast<const uint4*>(vp + t * D + 64 * c), vf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[8 * c + e] = fmaf(p, vf[e], acc[8 * c + e]);
                 }
@@ -340,7 +361,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
         }
         if (live) {
             const float inv = 1.f / l;
-            uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * E;
+            uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * 8;
 #pragma unroll
             for (int c = 0; c < V4; ++c) {
                 uint4 ov;
@@ -348,7 +369,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
                     ow[e] = (uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e] * inv) | ((uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e + 1] * inv) << 16);
-                *reinterpret_cast<uint4*>(op + 8 * c) = ov;
+                *reinterpret_cast<uint4*>(op + 64 * c) = ov;
             }
             if (sub == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
         }
