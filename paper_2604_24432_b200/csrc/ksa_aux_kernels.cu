@@ -129,37 +129,15 @@ __device__ __forceinline__ void summ_unpack(const uint4& raw, float* f)
     }
 }
 
+// The tasks [task_lo, task_hi) of one chunk and KV head by one warp; kp / vp point at the lane's elements of the
+// chunk's first K / V row (global or shared memory), kst / vst are the row strides in elements.
 template <int D>
-__global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
+__device__ __forceinline__ void summ_long_tasks(const KernelArgs& a, const uint16_t* kp, int64_t kst, const uint16_t* vp, int64_t vst,
+                                                int64_t row0, int hk, int G, int own, int task_lo, int task_hi, int lane)
 {
-    constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
+    constexpr int E = D / 8;
     constexpr int V4 = E / 8;
-    const bool ranged = a.r_seq >= 0;
-    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
-    const int hk = blockIdx.z;
-    const int G = a.Hq / a.Hkv;
-    const int tasks = a.m * G;
-    const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;
-    // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
-    const int j_first = ranged ? a.r_summ0 / a.m : 0;
-    const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
-    // consecutive warps take the task blocks of one chunk (they read the same K / V rows), then the next chunk's
-    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int j = j_first + (int)(gw / task_blocks);
-    if (j >= j_end) return;                                            // warp-uniform
-    const int task_lo = (int)(gw % task_blocks) * kSummTaskBlock;
-    const int task_hi = min(tasks, task_lo + kSummTaskBlock);
-    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
-    const int s = a.k + a.m;
-    const int own = (a.flags & 1u) ? 0 : 1;                            // a summary sees the chunk's summaries up to itself
-    const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
-    const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
-    const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
-    {
-        const int rows_seen = a.k + own * ((task_hi - 1) / G + 1);     // keys of the warp's last task
-        summ_prefetch_rows<D>(a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh, a.k_st, rows_seen, lane);
-        summ_prefetch_rows<D>(a.v + row0 * a.v_st + (int64_t)hk * a.v_sh, a.v_st, rows_seen, lane);
-    }
+    const int sub = lane & 7, grp = lane >> 3;
     for (int t0 = task_lo; t0 < task_hi; t0 += 4) {
         const int task = t0 + grp;
         const bool live = task < task_hi;
@@ -187,7 +165,7 @@ __global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
 #pragma unroll
                     for (int c = 0; c < V4; ++c) {
                         float kf[8];
-                        summ_unpack(*reinterpret_cast<const uint4*>(kp + (int64_t)(b0 + i) * a.k_st + 8 * c), kf);
+                        summ_unpack(*reinterpret_cast<const uint4*>(kp + (int64_t)(b0 + i) * kst + 8 * c), kf);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) dot = fmaf(qv[8 * c + e], kf[e], dot);
                     }
@@ -219,7 +197,7 @@ __global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
 #pragma unroll
                     for (int c = 0; c < V4; ++c) {
                         float vf[8];
-                        summ_unpack(*reinterpret_cast<const uint4*>(vp + (int64_t)(b0 + i) * a.v_st + 8 * c), vf);
+                        summ_unpack(*reinterpret_cast<const uint4*>(vp + (int64_t)(b0 + i) * vst + 8 * c), vf);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc[8 * c + e] = fmaf(p, vf[e], acc[8 * c + e]);
                     }
@@ -241,6 +219,77 @@ __global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
             if (sub == 0) a.lse[(int64_t)h * a.total_aug + qrow] = mx + __logf(l);
         }
     }
+}
+
+template <int D>
+__global__ void __launch_bounds__(256, 2) ksa_summary_kernel(KernelArgs a)
+{
+    constexpr int E = D / 8;                      // elements per lane: 16 (two 16-byte vectors) or 8 (one)
+    const bool ranged = a.r_seq >= 0;
+    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
+    const int hk = blockIdx.z;
+    const int G = a.Hq / a.Hkv;
+    const int tasks = a.m * G;
+    const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;
+    // whole chunks only: a range starts and ends on chunk boundaries of the summary stream
+    const int j_first = ranged ? a.r_summ0 / a.m : 0;
+    const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
+    // consecutive warps take the task blocks of one chunk (they read the same K / V rows), then the next chunk's
+    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int j = j_first + (int)(gw / task_blocks);
+    if (j >= j_end) return;                                            // warp-uniform
+    const int task_lo = (int)(gw % task_blocks) * kSummTaskBlock;
+    const int task_hi = min(tasks, task_lo + kSummTaskBlock);
+    const int lane = threadIdx.x & 31, sub = lane & 7;
+    const int s = a.k + a.m;
+    const int own = (a.flags & 1u) ? 0 : 1;                            // a summary sees the chunk's summaries up to itself
+    const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
+    const uint16_t* kp = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh + sub * E;
+    const uint16_t* vp = a.v + row0 * a.v_st + (int64_t)hk * a.v_sh + sub * E;
+    {
+        const int rows_seen = a.k + own * ((task_hi - 1) / G + 1);     // keys of the warp's last task
+        summ_prefetch_rows<D>(a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh, a.k_st, rows_seen, lane);
+        summ_prefetch_rows<D>(a.v + row0 * a.v_st + (int64_t)hk * a.v_sh, a.v_st, rows_seen, lane);
+    }
+    summ_long_tasks<D>(a, kp, a.k_st, vp, a.v_st, row0, hk, G, own, task_lo, task_hi, lane);
+}
+
+// The same with the chunk's K and V rows of the KV head staged in shared memory first (2 (k + m) D bf16, dynamic):
+// one block per (chunk, KV head), all its loads in flight at once, its warps take the chunk's task blocks in turn.
+template <int D>
+__global__ void __launch_bounds__(256, 2) ksa_summary_staged_kernel(KernelArgs a)
+{
+    constexpr int E = D / 8;
+    extern __shared__ __align__(16) uint16_t summ_smem[];
+    const bool ranged = a.r_seq >= 0;
+    const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
+    const int hk = blockIdx.z;
+    const int G = a.Hq / a.Hkv;
+    const int tasks = a.m * G;
+    const int j_first = ranged ? a.r_summ0 / a.m : 0;
+    const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
+    const int j = j_first + (int)blockIdx.x;
+    if (j >= j_end) return;                                            // block-uniform
+    const int s = a.k + a.m;
+    const int own = (a.flags & 1u) ? 0 : 1;
+    const int64_t row0 = sq.aug_off + (int64_t)j * s;
+    uint16_t* sK = summ_smem;
+    uint16_t* sV = summ_smem + s * D;
+    {
+        constexpr int vecs = D / 8;
+        const int total = s * vecs;
+        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+            const int rr = idx / vecs, vv = idx - rr * vecs;
+            const uint4 kx = *reinterpret_cast<const uint4*>(a.kx + (row0 + rr) * a.k_st + (int64_t)hk * a.k_sh + vv * 8);
+            const uint4 vx = *reinterpret_cast<const uint4*>(a.v + (row0 + rr) * a.v_st + (int64_t)hk * a.v_sh + vv * 8);
+            *reinterpret_cast<uint4*>(sK + rr * D + vv * 8) = kx;
+            *reinterpret_cast<uint4*>(sV + rr * D + vv * 8) = vx;
+        }
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, sub = lane & 7;
+    for (int task_lo = (int)(threadIdx.x >> 5) * kSummTaskBlock; task_lo < tasks; task_lo += (int)(blockDim.x >> 5) * kSummTaskBlock)
+        summ_long_tasks<D>(a, sK + sub * E, D, sV + sub * E, D, row0, hk, G, own, task_lo, min(tasks, task_lo + kSummTaskBlock), lane);
 }
 
 // Summary rows, short chunks (k + m <= kSummMaxKeys; the paper's layout has 9 keys per row).
@@ -392,9 +441,16 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
     } else {
         const int tasks = a.m * (a.Hq / a.Hkv);
         const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;
-        dim3 g3((unsigned)(((int64_t)max_chunks * task_blocks + 7) / 8), ny, (unsigned)a.Hkv);
-        if (a.D == 128) ksa_summary_kernel<128><<<g3, 256, 0, stream>>>(a);
-        else            ksa_summary_kernel<64><<<g3, 256, 0, stream>>>(a);
+        const size_t stage_bytes = (size_t)2 * (a.k + a.m) * a.D * sizeof(uint16_t);
+        if (stage_bytes <= 48 * 1024) {                   // the chunk's K / V rows fit the default dynamic window
+            dim3 g4((unsigned)max_chunks, ny, (unsigned)a.Hkv);
+            if (a.D == 128) ksa_summary_staged_kernel<128><<<g4, 256, stage_bytes, stream>>>(a);
+            else            ksa_summary_staged_kernel<64><<<g4, 256, stage_bytes, stream>>>(a);
+        } else {
+            dim3 g3((unsigned)(((int64_t)max_chunks * task_blocks + 7) / 8), ny, (unsigned)a.Hkv);
+            if (a.D == 128) ksa_summary_kernel<128><<<g3, 256, 0, stream>>>(a);
+            else            ksa_summary_kernel<64><<<g3, 256, 0, stream>>>(a);
+        }
     }
     return cudaGetLastError();
 }
