@@ -76,6 +76,8 @@ def test_full_size_layout_g_sampled(ctx):
     ([2048, 640, 1336], 8, 1, 16, 8, 2, 128),   # whole chunks everywhere: direct views, sequences not on tile boundaries
     ([1024, 320], 4, 2, 9, 4, 2, 64),      # direct views with m = 2, D = 64
     ([768], 128, 1, 2, 2, 1, 128),         # a chunk is a whole tile
+    ([1300], 200, 8, 1, 8, 1, 128),        # long chunks, 64 summary tasks per chunk (several task blocks, rows read from global memory)
+    ([900], 96, 4, 2, 4, 2, 64),           # head_dim 64, summary rows from staged chunk rows
 ])
 def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
     wl = synth.Workload("edge", 99, lens, Hq, Hkv, D)
