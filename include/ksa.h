@@ -64,6 +64,14 @@ extern "C" {
 /* Run the text rows through the plain CUDA-core cross-check kernel instead of the
  * tensor-core kernel.  Same schedule, same packed streams; slow; for debugging. */
 #define KSA_FLAG_REFERENCE_KERNEL    0x2u
+/* Run the text rows through the tensor-core kernel that keeps both query heads of a work
+ * item in ONE CTA, even where the CTA-pair kernel applies (head_dim 128, an even number of
+ * query heads per KV head; with whole-chunk lengths also k | 64 and m | 64).  Same results
+ * up to rounding order; for comparison and debugging. */
+#define KSA_FLAG_SINGLE_CTA_KERNEL   0x4u
+/* Run the text rows through the CTA-pair kernel wherever it applies (see above), whatever the
+ * library would pick by itself.  Ignored where it does not apply. */
+#define KSA_FLAG_CTA_PAIR_KERNEL     0x8u
 
 typedef struct ksa_ctx ksa_ctx;    /* opaque */
 
@@ -273,6 +281,10 @@ int ksa_clear_device_status(ksa_ctx* ctx);
 int ksa_last_cuda_error(const ksa_ctx* ctx);
 /* Kernels launched by this context since creation (pack + summary + text kernels). */
 int64_t ksa_launch_count(const ksa_ctx* ctx);
+/* The device as the text-row kernels use it: its SM count (the one-CTA kernel runs one persistent CTA
+ * on each) and the number of two-CTA clusters it runs at once (the CTA-pair kernel runs that many
+ * persistent pairs; 0 would switch that kernel off).  Either pointer may be NULL. */
+int ksa_device_info(ksa_ctx* ctx, int32_t* num_sms, int32_t* max_cta_pairs);
 /* Optional per-kernel timing: when enabled, ksa_attn_fwd records CUDA events on the
  * caller's stream before and after the text-row kernel (the dominant kernel).
  * ksa_text_kernel_ms waits for the most recent pair and returns the elapsed device

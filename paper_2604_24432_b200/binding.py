@@ -23,6 +23,8 @@ KSA_ERR_CUDA, KSA_ERR_TIMEOUT, KSA_ERR_NOMEM = -4, -5, -6
 KSA_PREP_NO_ROPE = 1
 KSA_FLAG_SUMMARY_TEXT_ONLY = 0x1
 KSA_FLAG_REFERENCE_KERNEL = 0x2
+KSA_FLAG_SINGLE_CTA_KERNEL = 0x4
+KSA_FLAG_CTA_PAIR_KERNEL = 0x8
 KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
 
 EXPORTS = [
@@ -30,7 +32,7 @@ EXPORTS = [
     "ksa_visible_pairs", "ksa_attn_fwd", "ksa_host_staging_bytes", "ksa_attn_fwd_host",
     "ksa_attn_fwd_noalloc", "ksa_bwd_workspace_bytes", "ksa_attn_bwd",
     "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
-    "ksa_last_cuda_error", "ksa_launch_count", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
+    "ksa_last_cuda_error", "ksa_launch_count", "ksa_device_info", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
     "ksa_strerror",
     "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
     "ksa_decode_text", "ksa_decode_summary",
@@ -117,6 +119,7 @@ def lib():
     L.ksa_last_cuda_error.argtypes = [vp]
     L.ksa_launch_count.restype = i64
     L.ksa_launch_count.argtypes = [vp]
+    L.ksa_device_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.ksa_enable_kernel_timing.argtypes = [vp, ctypes.c_int]
     L.ksa_text_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     cp = ctypes.POINTER(ksa_cache_params)
@@ -352,6 +355,12 @@ class Context:
 
     def launch_count(self) -> int:
         return int(lib().ksa_launch_count(self.handle))
+
+    def device_info(self):
+        """(SM count, two-CTA clusters the device runs at once)."""
+        n, c = ctypes.c_int32(), ctypes.c_int32()
+        _check(lib().ksa_device_info(self.handle, ctypes.byref(n), ctypes.byref(c)), "ksa_device_info")
+        return int(n.value), int(c.value)
 
     def enable_kernel_timing(self, on: bool = True):
         _check(lib().ksa_enable_kernel_timing(self.handle, int(on)), "ksa_enable_kernel_timing")

@@ -40,6 +40,9 @@ struct ksa_ctx {
     bool timing_valid = false;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     bool tc_ready = false;
+    bool pair_ready = false;          // CTA-pair text kernel set up on this device
+    int max_pairs = 0;                // clusters of two CTAs the device runs at once
+    bool bwd_ready = false, bwd_tc_ready = false;
     // host entry point: copy streams and per-chunk events of its upload / compute / download pipeline
     cudaStream_t s_in = nullptr, s_out = nullptr;
     std::vector<cudaEvent_t> ev_in, ev_done;
@@ -68,7 +71,7 @@ int validate(const ksa_params* p)
     if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
         return KSA_ERR_INVALID_ARG;
     if (p->reserved != 0) return KSA_ERR_INVALID_ARG;
-    if (p->flags & ~(KSA_FLAG_SUMMARY_TEXT_ONLY | KSA_FLAG_REFERENCE_KERNEL)) return KSA_ERR_INVALID_ARG;
+    if (p->flags & ~(KSA_FLAG_SUMMARY_TEXT_ONLY | KSA_FLAG_REFERENCE_KERNEL | KSA_FLAG_SINGLE_CTA_KERNEL | KSA_FLAG_CTA_PAIR_KERNEL)) return KSA_ERR_INVALID_ARG;
     if (!(p->softmax_scale > 0.f) || !std::isfinite(p->softmax_scale)) return KSA_ERR_INVALID_ARG;
     if (p->cu_text_lens[0] != 0) return KSA_ERR_INVALID_ARG;
     for (int b = 0; b < p->num_seqs; ++b)
@@ -434,6 +437,19 @@ extern "C" __attribute__((visibility("default"))) int ksa_clear_device_status(ks
 extern "C" __attribute__((visibility("default"))) int ksa_last_cuda_error(const ksa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 extern "C" __attribute__((visibility("default"))) int64_t ksa_launch_count(const ksa_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+extern "C" __attribute__((visibility("default"))) int ksa_device_info(ksa_ctx* ctx, int32_t* num_sms, int32_t* max_cta_pairs)
+{
+    if (!ctx) return KSA_ERR_INVALID_ARG;
+    if (!ctx->pair_ready) {
+        cudaError_t e = setup_text_pair(&ctx->max_pairs);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->pair_ready = true;
+    }
+    if (num_sms) *num_sms = ctx->num_sms;
+    if (max_cta_pairs) *max_cta_pairs = ctx->max_pairs;
+    return KSA_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) int ksa_enable_kernel_timing(ksa_ctx* ctx, int on)
 {
     if (!ctx) return KSA_ERR_INVALID_ARG;
@@ -534,11 +550,11 @@ extern "C" __attribute__((visibility("default"))) int ksa_schedule_dump(ksa_ctx*
 // ---------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------
-static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H)
+static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, int64_t rows, int H, int box_rows = kTileN)
 {
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -548,13 +564,13 @@ static int encode_stream_map(ksa_ctx* ctx, CUtensorMap* map, void* base, int D, 
 }
 
 // Chunked view of a caller tensor [rows, H, D] (element strides st, sh): dims {D, rows_per_chunk, chunks, H},
-// a box of 128 / rows_per_chunk chunks.  `base` points at the first row of the view's first chunk.
+// a box of box_rows / rows_per_chunk chunks.  `base` points at the first row of the view's first chunk.
 static int encode_chunk_map(ksa_ctx* ctx, CUtensorMap* map, const void* base, int D, int rows_per_chunk, int chunk_rows,
-                            int64_t chunks, int H, int64_t st, int64_t sh)
+                            int64_t chunks, int H, int64_t st, int64_t sh, int box_rows = kTileN)
 {
     const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows_per_chunk, (cuuint64_t)chunks, (cuuint64_t)H};
     const cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)chunk_rows * st * 2, (cuuint64_t)sh * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)rows_per_chunk, (cuuint32_t)(kTileN / rows_per_chunk), 1};
+    const cuuint32_t box[4] = {64, (cuuint32_t)rows_per_chunk, (cuuint32_t)(box_rows / rows_per_chunk), 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -591,15 +607,41 @@ static KernelArgs make_args(ksa_ctx* ctx, const ksa_params* p, const void* q, co
     return a;
 }
 
-// One-time kernel setup and the tensor maps of the packed streams (tensor-core path only).
-static int prepare_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, TextMaps& maps)
+// The tensor maps of a forward call: those of the one-CTA kernel, plus the two 64-key-row maps of the CTA-pair
+// kernel where that one applies.
+struct FwdMaps { TextMaps t; CUtensorMap kt_half, ks_half; bool pair = false; };
+
+// Which tensor-core kernel takes the text rows when the caller does not say (KSA_FLAG_SINGLE_CTA_KERNEL /
+// KSA_FLAG_CTA_PAIR_KERNEL): the faster one on the measured workloads.
+static constexpr bool kPairKernelByDefault = false;
+
+// The CTA-pair kernel takes work items of two query heads at head_dim 128; reading whole-chunk batches in place
+// it also needs half a K tile (64 rows) to be a whole number of chunks in both views.
+static bool pair_ok(const KernelArgs& a, uint32_t flags)
+{
+    if (flags & (KSA_FLAG_REFERENCE_KERNEL | KSA_FLAG_SINGLE_CTA_KERNEL)) return false;
+    if (a.D != 128 || ((a.Hq / a.Hkv) & 1)) return false;
+    if (a.direct && (64 % a.k != 0 || (a.m > 0 && 64 % a.m != 0))) return false;
+    return kPairKernelByDefault || (flags & KSA_FLAG_CTA_PAIR_KERNEL);
+}
+
+// One-time kernel setup and the tensor maps of the packed streams (tensor-core paths only).
+static int prepare_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, FwdMaps& fm)
 {
     if (flags & KSA_FLAG_REFERENCE_KERNEL) return KSA_OK;
+    TextMaps& maps = fm.t;
+    fm.pair = pair_ok(a, flags);
     if (!ctx->tc_ready) {
         cudaError_t e = setup_text_tc();
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         ctx->tc_ready = true;
     }
+    if (fm.pair && !ctx->pair_ready) {
+        cudaError_t e = setup_text_pair(&ctx->max_pairs);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->pair_ready = true;
+    }
+    if (fm.pair && ctx->max_pairs < 1) fm.pair = false;
     int rc;
     if (a.direct) {
         const int s_len = a.k + a.m;
@@ -607,25 +649,40 @@ static int prepare_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, TextM
         if ((rc = encode_chunk_map(ctx, &maps.qt, a.q, a.D, a.k, s_len, chunks, a.Hq, a.q_st, a.q_sh)) != KSA_OK) return rc;
         if ((rc = encode_chunk_map(ctx, &maps.kt, a.kx, a.D, a.k, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
         if ((rc = encode_chunk_map(ctx, &maps.vt, a.v, a.D, a.k, s_len, chunks, a.Hkv, a.v_st, a.v_sh)) != KSA_OK) return rc;
+        if (fm.pair && (rc = encode_chunk_map(ctx, &fm.kt_half, a.kx, a.D, a.k, s_len, chunks, a.Hkv, a.k_st, a.k_sh, 64)) != KSA_OK) return rc;
         if (a.m > 0) {      // summary rows start k rows into each chunk
             if ((rc = encode_chunk_map(ctx, &maps.ks, a.kx + (int64_t)a.k * a.k_st, a.D, a.m, s_len, chunks, a.Hkv, a.k_st, a.k_sh)) != KSA_OK) return rc;
+            if (fm.pair && (rc = encode_chunk_map(ctx, &fm.ks_half, a.kx + (int64_t)a.k * a.k_st, a.D, a.m, s_len, chunks, a.Hkv, a.k_st, a.k_sh, 64)) != KSA_OK) return rc;
             return encode_chunk_map(ctx, &maps.vs, a.v + (int64_t)a.k * a.v_st, a.D, a.m, s_len, chunks, a.Hkv, a.v_st, a.v_sh);
         }
         maps.ks = maps.kt; maps.vs = maps.vt;    // never used: no summary tiles are scheduled
+        fm.ks_half = fm.kt_half;
         return KSA_OK;
     }
     if ((rc = encode_stream_map(ctx, &maps.qt, a.qt, a.D, a.text_rows, a.Hq)) != KSA_OK) return rc;
     if ((rc = encode_stream_map(ctx, &maps.kt, a.kt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
     if ((rc = encode_stream_map(ctx, &maps.vt, a.vt, a.D, a.text_rows, a.Hkv)) != KSA_OK) return rc;
     if ((rc = encode_stream_map(ctx, &maps.ks, a.ks, a.D, a.summ_rows, a.Hkv)) != KSA_OK) return rc;
+    if (fm.pair) {
+        if ((rc = encode_stream_map(ctx, &fm.kt_half, a.kt, a.D, a.text_rows, a.Hkv, 64)) != KSA_OK) return rc;
+        if ((rc = encode_stream_map(ctx, &fm.ks_half, a.ks, a.D, a.summ_rows, a.Hkv, 64)) != KSA_OK) return rc;
+    }
     return encode_stream_map(ctx, &maps.vs, a.vs, a.D, a.summ_rows, a.Hkv);
 }
 
 // Text-row kernel over the work items a.work[0 .. a.num_work).
-static int launch_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, const TextMaps& maps, cudaStream_t stream)
+static int launch_text(ksa_ctx* ctx, const KernelArgs& a, uint32_t flags, const FwdMaps& fm, cudaStream_t stream)
 {
-    cudaError_t e = (flags & KSA_FLAG_REFERENCE_KERNEL) ? launch_text_ref(a, stream)
-                                                        : launch_text_tc(a, maps, ctx->num_sms, stream);
+    cudaError_t e;
+    if (flags & KSA_FLAG_REFERENCE_KERNEL) {
+        e = launch_text_ref(a, stream);
+    } else if (fm.pair) {
+        PairMaps pm;
+        pm.qt = fm.t.qt; pm.kt = fm.kt_half; pm.vt = fm.t.vt; pm.ks = fm.ks_half; pm.vs = fm.t.vs;
+        e = launch_text_pair(a, pm, ctx->max_pairs, stream);
+    } else {
+        e = launch_text_tc(a, fm.t, ctx->num_sms, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return KSA_OK;
@@ -658,7 +715,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd(ksa_ctx* ctx,
         ctx->launches += 1;
     }
     if (ctx->timing) cudaEventRecord(ctx->ev0, stream);
-    TextMaps maps;
+    FwdMaps maps;
     if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
     if ((rc = launch_text(ctx, a, p->flags, maps, stream)) != KSA_OK) return rc;
     if (ctx->timing) { cudaEventRecord(ctx->ev1, stream); ctx->timing_valid = true; }
@@ -754,7 +811,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_part(ksa_ctx*
     a.r_seq = -1;
     a.work = work_base + hs.chunks[c0].work_off;                         // the chunks' items follow one another in the list
     a.num_work = (int32_t)work_cnt;
-    TextMaps maps;
+    FwdMaps maps;
     if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
     return launch_text(ctx, a, p->flags, maps, stream);
 }
@@ -816,10 +873,9 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* ws = (char*)workspace;
     cudaError_t e;
-    static bool bwd_ready = false;
-    if (!bwd_ready) {
+    if (!ctx->bwd_ready) {            // the shared-memory opt-in is per device: kept per context
         if ((e = setup_bwd()) != cudaSuccess) return cuda_fail(ctx, e);
-        bwd_ready = true;
+        ctx->bwd_ready = true;
     }
     // packed streams of the forward pass (text Q, K, V and summary K, V) -- not needed when the tensor-core kernels
     // can read whole tiles straight from the caller's tensors (the no-pack case of the forward pass)
@@ -851,10 +907,9 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if (a.D == 128) {
         // text rows on the tcgen05 tensor cores, fed by TMA from the packed streams
-        static bool bwd_tc_ready = false;
-        if (!bwd_tc_ready) {
+        if (!ctx->bwd_tc_ready) {
             if ((e = setup_bwd_tc()) != cudaSuccess) return cuda_fail(ctx, e);
-            bwd_tc_ready = true;
+            ctx->bwd_tc_ready = true;
         }
         BwdMaps bm;
         if (direct) {
@@ -1036,7 +1091,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_host(ksa_ctx*
         ctx->ev_in.push_back(a0); ctx->ev_done.push_back(a1);
     }
     KernelArgs a = make_args(ctx, &pc, d + s.q, d + s.k, d + s.v, d + s.out, (float*)(d + s.lse), d + s.ws, wl);
-    TextMaps maps;
+    FwdMaps maps;
     if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
     // the copy-in stream starts after whatever the caller queued before this call
     if ((e = cudaEventRecord(ctx->ev_start, stream)) != cudaSuccess) return cuda_fail(ctx, e);

@@ -74,6 +74,10 @@ enum DeviceStatus : int32_t {
     kStatusWaitQFull = 1, kStatusWaitQEmpty = 2, kStatusWaitKvFull = 3, kStatusWaitKvEmpty = 4,
     kStatusWaitSFull = 5, kStatusWaitPFull = 6, kStatusWaitOFull = 7, kStatusWaitTest = 8,
     kStatusSmemLayout = 9,      // the dynamic shared memory window did not hold the 1024-byte aligned layout
+    kStatusWaitMaxPub = 10,     // CTA-pair kernel: the other softmax group's reference maximum
+    kStatusWaitRowSums = 11,    // CTA-pair kernel: the other softmax group's row sums
+    kStatusWaitPvDone = 12,     // CTA-pair kernel: completion of O += P V
+    kStatusWaitOEmpty = 13,     // CTA-pair kernel: the epilogue's read of O
 };
 
 }  // namespace ksa

@@ -27,6 +27,13 @@ cudaError_t launch_text_tc(const KernelArgs& a, const TextMaps& maps, int num_sm
 // One-time per-device setup (dynamic shared memory opt-in).
 cudaError_t setup_text_tc();
 
+// Text rows on CTA pairs (head_dim 128, work items of two query heads): same tensor maps, except that kt and ks
+// have boxes of 64 key rows ({64, 64, 1}; direct: {64, k, 64 / k, 1} and {64, m, 64 / m, 1}) -- each CTA of a pair
+// loads half of a K tile.  max_pairs = clusters of two CTAs the device runs at once (from setup_text_pair).
+struct PairMaps { CUtensorMap qt, kt, vt, ks, vs; };
+cudaError_t launch_text_pair(const KernelArgs& a, const PairMaps& maps, int max_pairs, cudaStream_t stream);
+cudaError_t setup_text_pair(int* max_pairs);
+
 // Q/K/V preparation upstream of the attention (position ids, interpolation at summary positions, rotary
 // embedding): one pass over the augmented rows.
 struct PrepArgs {

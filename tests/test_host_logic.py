@@ -114,6 +114,73 @@ def test_schedule_bit_exact_against_oracle_mask(lens, k, m, C):
                     assert (q0, ksa.KSA_STREAM_SUMMARY, u0) in seen
 
 
+def _check_query_tile(recs_tile, n, k, m, C, q0, TM=128):
+    """One query tile of one sequence against the oracle's explicit mask rows (every key position of the
+    sequence is put through the oracle's predicate): visited tiles <=> a visible pair, is_full <=> all visible,
+    nothing visited twice."""
+    tp, sp, L = None, None, orc.aug_len(n, k, m)
+    s_len = k + m
+    J = n // k
+    i = np.arange(n, dtype=np.int64)
+    tpos = np.where(i < J * k, (i // k) * s_len + i % k, J * s_len + (i - J * k))          # Eq. 1
+    u = np.arange(J * m, dtype=np.int64)
+    spos = (u // max(m, 1)) * s_len + k + u % max(m, 1) if m else np.zeros(0, np.int64)
+    q1 = min(n, q0 + TM)
+    rows = np.stack([orc.mask_row(n, k, m, C, int(tpos[r])) for r in range(q0, q1)]).astype(bool)
+    vis_t, vis_s = rows[:, tpos], rows[:, spos]
+    assert rows.sum() == vis_t.sum() + vis_s.sum()
+    want = {}
+    for a0 in range(0, n, TM):
+        sub = vis_t[:, a0:a0 + TM]
+        if sub.any():
+            want[(ksa.KSA_STREAM_TEXT, a0)] = (min(TM, n - a0), bool(sub.all()))
+    for u0 in range(0, len(spos), TM):
+        sub = vis_s[:, u0:u0 + TM]
+        if sub.any():
+            want[(ksa.KSA_STREAM_SUMMARY, u0)] = (min(TM, len(spos) - u0), bool(sub.all()))
+    got = {}
+    for r in recs_tile:
+        key = (int(r["kv_stream"]), int(r["kv_row0"]))
+        assert key not in got, key
+        assert int(r["q_rows"]) == q1 - q0
+        got[key] = (int(r["kv_rows"]), bool(r["is_full"]))
+    assert got == want
+
+
+@pytest.mark.parametrize("layout", ["P", "G"])
+def test_schedule_bit_exact_8k_workload(layout):
+    """The 8K workload, every query tile, both layouts."""
+    from paper_2604_24432_b200 import synth
+    wl, lay = synth.WORKLOADS["8k"], {"P": synth.LAYOUT_P, "G": synth.LAYOUT_G}[layout]
+    prob = ksa.Problem(wl.text_lens, lay.k, lay.m, lay.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    recs = ksa.schedule_dump(prob)
+    n = wl.text_lens[0]
+    for q0 in range(0, n, 128):
+        _check_query_tile(recs[(recs["seq"] == 0) & (recs["q_row0"] == q0)], n, lay.k, lay.m, lay.C, q0)
+    assert len(recs) == sum(len(recs[(recs["seq"] == 0) & (recs["q_row0"] == q0)]) for q0 in range(0, n, 128))
+
+
+@pytest.mark.parametrize("name,layout", [("tiny", "P"), ("tiny", "G"), ("32k", "P"), ("32k", "G"), ("128k", "P"), ("128k", "G"),
+                                         ("varlen", "P"), ("varlen", "G")])
+def test_schedule_bit_exact_workloads_sampled(name, layout):
+    """The other workloads at full size: in every sequence the first and last query tiles, the tiles on either side of
+    the point where the window stops reaching token 0, the tile in the middle and seeded random tiles, each checked
+    tile by tile against the oracle's mask rows."""
+    from paper_2604_24432_b200 import synth
+    wl, lay = synth.WORKLOADS[name], {"P": synth.LAYOUT_P, "G": synth.LAYOUT_G}[layout]
+    prob = ksa.Problem(wl.text_lens, lay.k, lay.m, lay.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    recs = ksa.schedule_dump(prob)
+    rng = np.random.default_rng(7)
+    for b, n in enumerate(wl.text_lens):
+        n_t = (n + 127) // 128
+        edge = (lay.C * lay.k) // 128                      # first tile whose rows start to lose token 0
+        tiles = {0, n_t - 1, max(0, n_t - 2), min(n_t - 1, edge), min(n_t - 1, edge + 1), max(0, min(n_t - 1, edge - 1)), n_t // 2}
+        tiles |= set(int(t) for t in rng.integers(0, n_t, size=2 if len(wl.text_lens) > 2 else 4))
+        rb = recs[recs["seq"] == b]
+        for t in sorted(tiles):
+            _check_query_tile(rb[rb["q_row0"] == t * 128], n, lay.k, lay.m, lay.C, t * 128)
+
+
 def test_schedule_tile_counts_128k():
     """Per-head visited tiles of the 128K workload: 65,024 summary + 9,180 text tiles."""
     prob = ksa.Problem([131072], 8, 1, 128, 32, 4, 128, 0.0883)
