@@ -243,8 +243,14 @@ int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, cons
  * CURRENT device; results are identical to ksa_attn_fwd's.
  * Limits and behaviour:
  *   - Problems whose scratch exceeds the array are rejected with KSA_ERR_WORKSPACE
- *     before anything is enqueued (scratch = 256 B + 48 B per sequence + 48 B per work
- *     item + ksa_workspace_bytes(p)).
+ *     before anything is enqueued.  This entry point ALWAYS packs the text and summary rows
+ *     into dense streams (ksa_attn_fwd skips that for whole-chunk batches and then reports
+ *     a 256-byte workspace, which is NOT what counts here).  Scratch = 1,280 B + 48 B per
+ *     sequence + 48 B per work item (query tiles x pairs of query heads; single heads if
+ *     the group size is odd) + the packed streams: 2 * head_dim bytes x
+ *     [(num_q_heads + 2 * num_kv_heads) x text rows + 2 * num_kv_heads x summary rows],
+ *     each sequence's rows rounded up to a multiple of 128.  Of the five benchmark
+ *     workloads only the 1,024-token one fits.
  *   - The first call on each device resolves the array's device address and opts the
  *     kernels into their shared-memory size; make that first call outside any stream
  *     capture.
@@ -258,6 +264,13 @@ int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, cons
 #define KSA_NOALLOC_MAX_SCRATCH_BYTES (32u * 1024u * 1024u)
 int ksa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
                          const ksa_params* p, void* cuda_stream);
+/* The status word of ksa_attn_fwd_noalloc's bounded waits on the CURRENT device (it lives in the
+ * fixed array, so no context is needed): a blocking 4-byte copy, no allocation.  *status = 0 and
+ * KSA_OK if no wait gave up since the last call started (each call re-zeroes the word before its
+ * kernels run, so read it after the stream has finished and before the next call); otherwise the
+ * code of the first wait that gave up, and KSA_ERR_TIMEOUT -- out and lse of that call are then
+ * not valid.  (No counterpart in the paper.) */
+int ksa_noalloc_last_device_status(int32_t* status);
 
 /* ---- schedule inspection ------------------------------------------------------------ */
 /*
@@ -272,9 +285,20 @@ int ksa_schedule_dump(ksa_ctx* ctx, const ksa_params* p, ksa_tile_rec* recs, int
 
 /* ---- diagnostics -------------------------------------------------------------------- */
 /* Reads (with a blocking copy) the device status word written by bounded waits:
- * 0 = no wait ever gave up; otherwise a code naming the first wait that did (9: a kernel found
- * that its shared-memory layout does not fit the window it was given, and did nothing). */
+ * 0 = no wait gave up since the word was last cleared (returns KSA_OK); otherwise a code naming
+ * the first wait that did (9: a kernel found that its shared-memory layout does not fit the
+ * window it was given, and did nothing) and the call returns KSA_ERR_TIMEOUT: the results of
+ * the calls enqueued since the last clear are not valid.  Every device-side wait of the library
+ * is bounded (about a second); a kernel whose wait gives up leaves its loops, waits (bounded)
+ * for its copies in flight, frees its TMEM and returns, so the context stays usable. */
 int ksa_last_device_status(ksa_ctx* ctx, int32_t* status);
+/* Self-test of that path (no counterpart in the paper): a one-warp kernel waits with the library's
+ * bounded-wait helper, limited to limit_cycles SM cycles (1 .. 2^31), on a barrier that nothing
+ * arrives at.  Afterwards ksa_last_device_status reports code 8 and KSA_ERR_TIMEOUT, and
+ * report5_device (DEVICE, five int32) holds {first wait succeeded (0 expected), second wait
+ * succeeded (0: it saw the abort flag), abort flag (1), kilo-cycles in the first wait, in the second}.
+ * Asynchronous on cuda_stream. */
+int ksa_selftest_bounded_wait(ksa_ctx* ctx, int64_t limit_cycles, int32_t* report5_device, void* cuda_stream);
 /* Clears the device status word (blocking copy). */
 int ksa_clear_device_status(ksa_ctx* ctx);
 /* Last cudaError_t / CUresult seen by this context (0 = none). */

@@ -30,8 +30,8 @@ KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
 EXPORTS = [
     "ksa_create", "ksa_destroy", "ksa_aug_len", "ksa_total_aug_len", "ksa_workspace_bytes",
     "ksa_visible_pairs", "ksa_attn_fwd", "ksa_host_staging_bytes", "ksa_attn_fwd_host",
-    "ksa_attn_fwd_noalloc", "ksa_bwd_workspace_bytes", "ksa_attn_bwd",
-    "ksa_schedule_dump", "ksa_last_device_status", "ksa_clear_device_status",
+    "ksa_attn_fwd_noalloc", "ksa_noalloc_last_device_status", "ksa_bwd_workspace_bytes", "ksa_attn_bwd",
+    "ksa_schedule_dump", "ksa_selftest_bounded_wait", "ksa_last_device_status", "ksa_clear_device_status",
     "ksa_last_cuda_error", "ksa_launch_count", "ksa_device_info", "ksa_enable_kernel_timing", "ksa_text_kernel_ms",
     "ksa_strerror",
     "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
@@ -104,6 +104,7 @@ def lib():
     L.ksa_host_staging_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, pp, vp]
+    L.ksa_noalloc_last_device_status.argtypes = [ctypes.POINTER(i32)]
     L.ksa_bwd_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
     L.ksa_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_part_rows.argtypes = [vp, pp, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -115,6 +116,7 @@ def lib():
     L.ksa_qkv_prepare.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, pp, vp]
     L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
     L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.ksa_selftest_bounded_wait.argtypes = [vp, i64, vp, vp]
     L.ksa_clear_device_status.argtypes = [vp]
     L.ksa_last_cuda_error.argtypes = [vp]
     L.ksa_launch_count.restype = i64
@@ -344,8 +346,19 @@ class Context:
 
     def device_status(self) -> int:
         s = ctypes.c_int32()
-        _check(lib().ksa_last_device_status(self.handle, ctypes.byref(s)), "ksa_last_device_status")
+        rc = lib().ksa_last_device_status(self.handle, ctypes.byref(s))
+        if rc not in (KSA_OK, KSA_ERR_TIMEOUT):          # KSA_ERR_TIMEOUT: the status word is non-zero, returned below
+            _check(rc, "ksa_last_device_status")
         return int(s.value)
+
+    def device_status_rc(self) -> int:
+        """The return code of ksa_last_device_status itself (KSA_OK or KSA_ERR_TIMEOUT)."""
+        s = ctypes.c_int32()
+        return int(lib().ksa_last_device_status(self.handle, ctypes.byref(s)))
+
+    def selftest_bounded_wait(self, limit_cycles: int, report, stream: Optional[int] = None):
+        _check(lib().ksa_selftest_bounded_wait(self.handle, int(limit_cycles), report.data_ptr(), stream),
+               "ksa_selftest_bounded_wait")
 
     def clear_device_status(self):
         _check(lib().ksa_clear_device_status(self.handle), "ksa_clear_device_status")
@@ -372,6 +385,15 @@ class Context:
 
 
 NOALLOC_MAX_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def noalloc_device_status() -> int:
+    """Status word of the allocation-free entry point on the current device (0 = no wait gave up)."""
+    st = ctypes.c_int32()
+    rc = lib().ksa_noalloc_last_device_status(ctypes.byref(st))
+    if rc not in (KSA_OK, KSA_ERR_TIMEOUT):
+        _check(rc, "ksa_noalloc_last_device_status")
+    return int(st.value)
 
 
 def attn_fwd_noalloc(prob: Problem, q, k, v, out, lse, stream: Optional[int] = None):

@@ -42,7 +42,7 @@ struct ksa_ctx {
     bool tc_ready = false;
     bool pair_ready = false;          // CTA-pair text kernel set up on this device
     int max_pairs = 0;                // clusters of two CTAs the device runs at once
-    bool bwd_ready = false, bwd_tc_ready = false;
+    bool bwd_ready = false, bwd_tc_ready = false, decode_ready = false;
     // host entry point: copy streams and per-chunk events of its upload / compute / download pipeline
     cudaStream_t s_in = nullptr, s_out = nullptr;
     std::vector<cudaEvent_t> ev_in, ev_done;
@@ -59,6 +59,7 @@ int32_t* ksa_ctx_status_word(ksa_ctx* ctx) { return ctx->d_status; }
 int ksa_ctx_num_sms(const ksa_ctx* ctx) { return ctx->num_sms; }
 void ksa_ctx_add_launches(ksa_ctx* ctx, int n) { ctx->launches += n; }
 int ksa_ctx_cuda_fail(ksa_ctx* ctx, int cuda_error) { return cuda_fail(ctx, (cudaError_t)cuda_error); }
+bool* ksa_ctx_decode_ready(ksa_ctx* ctx) { return &ctx->decode_ready; }
 
 // ---------------------------------------------------------------------------------------
 // validation and layout
@@ -424,7 +425,8 @@ extern "C" __attribute__((visibility("default"))) int ksa_last_device_status(ksa
 {
     if (!ctx || !status) return KSA_ERR_INVALID_ARG;
     cudaError_t e = cudaMemcpy(status, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost);
-    return e == cudaSuccess ? KSA_OK : cuda_fail(ctx, e);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return *status != 0 ? KSA_ERR_TIMEOUT : KSA_OK;
 }
 
 extern "C" __attribute__((visibility("default"))) int ksa_clear_device_status(ksa_ctx* ctx)

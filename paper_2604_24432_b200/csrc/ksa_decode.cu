@@ -546,7 +546,7 @@ static int decode_step(ksa_ctx* ctx, int summary_step, void* kcache, void* vcach
     a.summary_step = summary_step;
     a.flags = p->flags;
     a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
-    static bool attr_done = false;
+    bool& attr_done = *ksa_ctx_decode_ready(ctx);         // per context: the opt-in is a per-device setting
     const int smem = kDecStages * 2 * kDecTile * a.D * 2;
     cudaError_t e;
     if (!attr_done) {

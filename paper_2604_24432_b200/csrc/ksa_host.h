@@ -46,3 +46,4 @@ int32_t* ksa_ctx_status_word(ksa_ctx* ctx);                 // device status wor
 int ksa_ctx_num_sms(const ksa_ctx* ctx);
 void ksa_ctx_add_launches(ksa_ctx* ctx, int n);
 int ksa_ctx_cuda_fail(ksa_ctx* ctx, int cuda_error);        // records the error, returns KSA_ERR_CUDA
+bool* ksa_ctx_decode_ready(ksa_ctx* ctx);                   // the decode kernels' shared-memory opt-in was done on this context's device

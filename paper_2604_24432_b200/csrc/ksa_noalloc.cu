@@ -82,6 +82,20 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+// The status word of the bounded waits is the first word of the scratch array; no context is involved, so it has
+// its own reader (a blocking 4-byte copy: allocates nothing).
+extern "C" __attribute__((visibility("default")))
+int ksa_noalloc_last_device_status(int32_t* status)
+{
+    if (!status) return KSA_ERR_INVALID_ARG;
+    int dev = -1;
+    DeviceSetup* setup = nullptr;
+    int rc = setup_current_device(&dev, &setup);
+    if (rc != KSA_OK) return rc;
+    if (cudaMemcpy(status, setup->scratch, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return KSA_ERR_CUDA;
+    return *status != 0 ? KSA_ERR_TIMEOUT : KSA_OK;
+}
+
 extern "C" __attribute__((visibility("default")))
 int ksa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
                          const ksa_params* p, void* cuda_stream)

@@ -54,7 +54,7 @@ constexpr int kRegsOther = 72;
 static_assert(8 * kRegsSoftmax + 4 * kRegsOther <= 12 * ((65536 / kThreads) / 8 * 8), "register hand-over exceeds the CTA's allocation");
 constexpr int kQkWarp = 11, kPvWarp = 9, kKProdWarp = 8, kVProdWarp = 10;
 #ifndef KSA_RESCALE_T
-#define KSA_RESCALE_T 20.0f
+#define KSA_RESCALE_T 12.0f
 #endif
 constexpr float kRescaleThreshold = KSA_RESCALE_T;
 constexpr int D = 128;
@@ -180,6 +180,12 @@ __device__ __forceinline__ bool wait_tagged(uint32_t addr, uint32_t tag, float& 
     for (uint32_t it = 0;; ++it) {
         asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(addr) : "memory");
         if (b == tag) { v = __uint_as_float(a); return true; }
+#if !defined(KSA_TAG_SLEEP_NS) || KSA_TAG_SLEEP_NS > 0
+#ifndef KSA_TAG_SLEEP_NS
+#define KSA_TAG_SLEEP_NS 32
+#endif
+        __nanosleep(KSA_TAG_SLEEP_NS);        // a tight read loop only burns issue slots and power next to the working warps
+#endif
         if (it == 0) t0 = clock64();
         if ((it & 63u) == 63u) {
             if (lds_u32(c.abort_addr) != 0u) return false;

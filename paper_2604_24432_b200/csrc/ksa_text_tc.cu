@@ -30,6 +30,7 @@
 
 #include "ksa_launch.h"
 #include "ksa_ptx.cuh"
+#include "ksa_wait.cuh"
 
 namespace ksa {
 
@@ -62,7 +63,11 @@ constexpr int kRegsOther = 72;            // ... of the producer / MMA warpgroup
 static_assert(8 * kRegsSoftmax + 4 * kRegsOther <= 12 * ((65536 / 384) / 8 * 8), "register hand-over exceeds the CTA's allocation");
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr float kRescaleThreshold = 8.0f;    // log2 units: P stays below 2^8
+// log2 units: P stays below 2^12.  A small threshold costs rescales of O: with 1 % of the keys four times larger (the 128k
+// workload) some row of nearly every warp outgrew 2^8 once or twice per work item.  Measured at 128k: 8 -> 1,032,
+// 12 -> 1,047, 20 -> 1,058 TFLOP/s, but the error against the fp64 oracle grows with it (mean |err| 5.6e-4, 5.9e-4,
+// 6.2e-4; at 20 one sampled element of the 64 + 8 layout left the 2e-2 bound), so 12 it is.
+constexpr float kRescaleThreshold = 12.0f;
 
 template <int D>
 struct TcCfg {
@@ -87,35 +92,6 @@ struct TcShared {
     uint32_t bars;        // smem address of barrier 0
     uint32_t abort_addr;  // smem address of the abort flag
 };
-
-__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t v)
-{
-    asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-
-// Bounded wait.  Returns false if the wait gave up or the CTA is aborting.
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, uint32_t abort_addr, int32_t* status, int code)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (ld_shared_u32(abort_addr) != 0u) return false;
-            if (clock64() - t0 > (1ll << 31)) {
-                atomicCAS(status, 0, code);
-                st_shared_u32(abort_addr, 1u);
-                return false;
-            }
-        }
-    }
-}
 
 template <int D>
 __global__ void __launch_bounds__(kThreadsTc, 1)
@@ -327,7 +303,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
         // instruction stream.  Every thread follows the ring position (two stages per key tile).
         int rel_stage = 0;
         auto release_next = [&]() {
-            mbar_arrive(kv_empty(rel_stage));
+            mbar_arrive_relaxed(kv_empty(rel_stage));
             if (++rel_stage == Cfg::kStages) rel_stage = 0;
         };
         for (int r = 0; alive; ++r) {
@@ -355,7 +331,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 if (releaser) {
                     if (j > 0) release_next();                   // V(j-1)
                     release_next();                              // K(j)
-                    if (j == T - 1) mbar_arrive(bar(BAR_QEMPTY));
+                    if (j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
                 } else if ((tid & 127) == 0) {
                     rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
                 }
@@ -449,8 +425,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 }
                 tc_wait_st();
                 tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
+                if (lane == 0) mbar_arrive_relaxed(bar(BAR_PFULL + t));
                 if (row == 0) KSA_TR(1 + t, 6);
                 if (lane == 0 && row != 0) KSA_TR(4 + warp, 6);
             }
