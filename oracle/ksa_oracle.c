@@ -315,3 +315,138 @@ int ksa_oracle_bwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v, con
     }
     return 0;
 }
+
+/* The same gradients on a SAMPLE of rows, for inputs too long to differentiate in full:
+ *   dq of the query rows q_rows[0..nq)   (global augmented rows; dq of a row only involves that row's own weights);
+ *   dk, dv of the key rows k_rows[0..nk) (the sums over every query row of the same sequence that sees the key).
+ * Same arithmetic as ksa_oracle_bwd, term by term; every query row that sees a sampled key still gets its complete
+ * softmax over its explicit mask row.  Outputs: dq [nq, Hq, D], dk and dv [nk, Hkv, D]. */
+int ksa_oracle_bwd_rows(const uint16_t* q, const uint16_t* kk, const uint16_t* v, const uint16_t* dout,
+                        int32_t num_seqs, const int32_t* cu_text_lens,
+                        int32_t k, int32_t m, int32_t C,
+                        int32_t Hq, int32_t Hkv, int32_t D, double scale, uint32_t flags,
+                        const int64_t* q_rows, int64_t nq, double* dq,
+                        const int64_t* k_rows, int64_t nk, double* dk, double* dv)
+{
+    if (!q || !kk || !v || !dout || !cu_text_lens) return -1;
+    if ((nq > 0 && (!q_rows || !dq)) || (nk > 0 && (!k_rows || !dk || !dv)) || nq < 0 || nk < 0) return -1;
+    if (num_seqs < 1 || k < 1 || m < 0 || C < 0 || Hq < 1 || Hkv < 1 || D < 1 || Hq % Hkv != 0) return -1;
+    const int32_t G = Hq / Hkv;
+    int64_t total_aug = 0, max_L = 1;
+    for (int32_t b = 0; b < num_seqs; ++b) {
+        int64_t L = ksa_oracle_aug_len((int64_t)cu_text_lens[b + 1] - cu_text_lens[b], k, m);
+        if (L < 0) return -1;
+        total_aug += L;
+        if (L > max_L) max_L = L;
+    }
+    for (int64_t r = 0; r < nq; ++r) if (q_rows[r] < 0 || q_rows[r] >= total_aug) return -1;
+    for (int64_t r = 0; r < nk; ++r) if (k_rows[r] < 0 || k_rows[r] >= total_aug) return -1;
+    if (nq > 0) memset(dq, 0, sizeof(double) * (size_t)nq * Hq * D);
+    if (nk > 0) { memset(dk, 0, sizeof(double) * (size_t)nk * Hkv * D); memset(dv, 0, sizeof(double) * (size_t)nk * Hkv * D); }
+
+    /* ---- dq of the sampled query rows ---- */
+#pragma omp parallel
+    {
+        uint8_t* mask = (uint8_t*)malloc((size_t)max_L);
+        double* p = (double*)malloc(sizeof(double) * (size_t)max_L);
+        double* o = (double*)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < nq; ++r) {
+            const int64_t g = q_rows[r];
+            int64_t base = 0, n = 0, L = 0;
+            for (int32_t b = 0; b < num_seqs; ++b) {              /* the sequence that holds row g */
+                n = (int64_t)cu_text_lens[b + 1] - cu_text_lens[b];
+                L = ksa_oracle_aug_len(n, k, m);
+                if (g < base + L) break;
+                base += L;
+            }
+            ksa_oracle_mask_row(n, k, m, C, flags, g - base, mask);
+            for (int32_t h = 0; h < Hq; ++h) {
+                const int32_t hk = h / G;
+                row_weights(q, kk, v, base, L, g, h, hk, Hq, Hkv, D, scale, mask, p, o);
+                const uint16_t* drow = dout + ((size_t)g * Hq + h) * (size_t)D;
+                double delta = 0.0;
+                for (int32_t d = 0; d < D; ++d) delta += bf16_to_double(drow[d]) * o[d];
+                double* dqrow = dq + ((size_t)r * Hq + h) * (size_t)D;
+                for (int64_t pk = 0; pk < L; ++pk) {
+                    if (!mask[pk]) continue;
+                    const size_t kvoff = ((size_t)(base + pk) * Hkv + hk) * (size_t)D;
+                    double dP = 0.0;
+                    for (int32_t d = 0; d < D; ++d) dP += bf16_to_double(drow[d]) * bf16_to_double(v[kvoff + d]);
+                    const double dS = p[pk] * (dP - delta);
+                    for (int32_t d = 0; d < D; ++d) dqrow[d] += scale * dS * bf16_to_double(kk[kvoff + d]);
+                }
+            }
+        }
+        free(mask); free(p); free(o);
+    }
+    if (nk == 0) return 0;
+
+    /* ---- dk, dv of the sampled key rows: every query row of the key's sequence is asked whether it sees the key ---- */
+    int nthreads = 1;
+#ifdef _OPENMP
+    nthreads = omp_get_max_threads();
+#endif
+    const size_t acc_len = (size_t)nk * Hkv * D;
+    double* part_k = (double*)calloc((size_t)nthreads * acc_len, sizeof(double));
+    double* part_v = (double*)calloc((size_t)nthreads * acc_len, sizeof(double));
+    if (!part_k || !part_v) { free(part_k); free(part_v); return -2; }
+    int64_t base = 0;
+    for (int32_t b = 0; b < num_seqs; ++b) {
+        const int64_t n = (int64_t)cu_text_lens[b + 1] - cu_text_lens[b];
+        const int64_t L = ksa_oracle_aug_len(n, k, m);
+        int64_t in_seq = 0;
+        for (int64_t r = 0; r < nk; ++r) if (k_rows[r] >= base && k_rows[r] < base + L) ++in_seq;
+        if (in_seq > 0) {
+#pragma omp parallel
+            {
+                int tid = 0;
+#ifdef _OPENMP
+                tid = omp_get_thread_num();
+#endif
+                double* ak = part_k + (size_t)tid * acc_len;
+                double* av = part_v + (size_t)tid * acc_len;
+                uint8_t* mask = (uint8_t*)malloc((size_t)max_L);
+                double* p = (double*)malloc(sizeof(double) * (size_t)max_L);
+                double* o = (double*)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 16)
+                for (int64_t pq = 0; pq < L; ++pq) {
+                    ksa_oracle_mask_row(n, k, m, C, flags, pq, mask);
+                    int any = 0;
+                    for (int64_t r = 0; r < nk && !any; ++r)
+                        if (k_rows[r] >= base && k_rows[r] < base + L && mask[k_rows[r] - base]) any = 1;
+                    if (!any) continue;
+                    const int64_t g = base + pq;
+                    for (int32_t h = 0; h < Hq; ++h) {
+                        const int32_t hk = h / G;
+                        row_weights(q, kk, v, base, L, g, h, hk, Hq, Hkv, D, scale, mask, p, o);
+                        const uint16_t* qrow = q + ((size_t)g * Hq + h) * (size_t)D;
+                        const uint16_t* drow = dout + ((size_t)g * Hq + h) * (size_t)D;
+                        double delta = 0.0;
+                        for (int32_t d = 0; d < D; ++d) delta += bf16_to_double(drow[d]) * o[d];
+                        for (int64_t r = 0; r < nk; ++r) {
+                            const int64_t pk = k_rows[r] - base;
+                            if (pk < 0 || pk >= L || !mask[pk]) continue;
+                            const size_t kvoff = ((size_t)(base + pk) * Hkv + hk) * (size_t)D;
+                            double dP = 0.0;
+                            for (int32_t d = 0; d < D; ++d) dP += bf16_to_double(drow[d]) * bf16_to_double(v[kvoff + d]);
+                            const double dS = p[pk] * (dP - delta);
+                            double* akr = ak + ((size_t)r * Hkv + hk) * (size_t)D;
+                            double* avr = av + ((size_t)r * Hkv + hk) * (size_t)D;
+                            for (int32_t d = 0; d < D; ++d) {
+                                avr[d] += p[pk] * bf16_to_double(drow[d]);
+                                akr[d] += scale * dS * bf16_to_double(qrow[d]);
+                            }
+                        }
+                    }
+                }
+                free(mask); free(p); free(o);
+            }
+        }
+        base += L;
+    }
+    for (int t = 0; t < nthreads; ++t)
+        for (size_t e = 0; e < acc_len; ++e) { dk[e] += part_k[(size_t)t * acc_len + e]; dv[e] += part_v[(size_t)t * acc_len + e]; }
+    free(part_k); free(part_v);
+    return 0;
+}

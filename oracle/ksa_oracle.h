@@ -106,6 +106,17 @@ int ksa_oracle_bwd(const uint16_t* q, const uint16_t* kk, const uint16_t* v, con
                    int32_t Hq, int32_t Hkv, int32_t D, double scale, uint32_t flags,
                    double* dq, double* dk, double* dv);
 
+/* The same gradients on a sample of rows (for inputs too long to differentiate in full): dq [nq, Hq, D] of the
+ * query rows q_rows (global augmented rows), dk and dv [nk, Hkv, D] of the key rows k_rows -- the latter summed
+ * over every query row of the key's sequence that sees the key, each with its complete softmax over its explicit
+ * mask row.  Same arithmetic as ksa_oracle_bwd.  Returns 0, -1 on bad arguments, -2 if out of memory. */
+int ksa_oracle_bwd_rows(const uint16_t* q, const uint16_t* kk, const uint16_t* v, const uint16_t* dout,
+                        int32_t num_seqs, const int32_t* cu_text_lens,
+                        int32_t k, int32_t m, int32_t C,
+                        int32_t Hq, int32_t Hkv, int32_t D, double scale, uint32_t flags,
+                        const int64_t* q_rows, int64_t nq, double* dq,
+                        const int64_t* k_rows, int64_t nk, double* dk, double* dv);
+
 /* Threads the OpenMP loops will use. */
 int ksa_oracle_num_threads(void);
 

@@ -64,6 +64,8 @@ def _load():
     lib.ksa_oracle_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, i32,
                                    ctypes.c_double, u32, vp, i64, vp, vp, vp]
     lib.ksa_oracle_bwd.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, i32, ctypes.c_double, u32, vp, vp, vp]
+    lib.ksa_oracle_bwd_rows.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, i32, ctypes.c_double, u32,
+                                        vp, i64, vp, vp, i64, vp, vp]
     lib.ksa_oracle_num_threads.restype = ctypes.c_int
     _lib = lib
     return lib
@@ -171,4 +173,29 @@ def bwd(q_bits, k_bits, v_bits, dout_bits, text_lens, k, m, C, scale, flags=0):
                             dq.ctypes.data, dk.ctypes.data, dv.ctypes.data)
     if rc != 0:
         raise ValueError("ksa_oracle_bwd: bad arguments")
+    return dq, dk, dv
+
+
+def bwd_rows(q_bits, k_bits, v_bits, dout_bits, text_lens, k, m, C, scale, q_rows, k_rows, flags=0):
+    """Gradients on a sample: dq [len(q_rows), Hq, D] of the query rows and dk, dv [len(k_rows), Hkv, D] of the key rows
+    (global augmented row indices), all float64."""
+    lib = _load()
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    k_bits = np.ascontiguousarray(k_bits, dtype=np.uint16)
+    v_bits = np.ascontiguousarray(v_bits, dtype=np.uint16)
+    dout_bits = np.ascontiguousarray(dout_bits, dtype=np.uint16)
+    total, Hq, D = q_bits.shape
+    Hkv = k_bits.shape[1]
+    cu = np.concatenate([[0], np.cumsum(np.asarray(text_lens, dtype=np.int64))]).astype(np.int32)
+    q_rows = np.ascontiguousarray(q_rows, dtype=np.int64)
+    k_rows = np.ascontiguousarray(k_rows, dtype=np.int64)
+    dq = np.empty((len(q_rows), Hq, D), dtype=np.float64)
+    dk = np.empty((len(k_rows), Hkv, D), dtype=np.float64)
+    dv = np.empty((len(k_rows), Hkv, D), dtype=np.float64)
+    rc = lib.ksa_oracle_bwd_rows(q_bits.ctypes.data, k_bits.ctypes.data, v_bits.ctypes.data, dout_bits.ctypes.data,
+                                 len(text_lens), cu.ctypes.data, k, m, C, Hq, Hkv, D, float(scale), flags,
+                                 q_rows.ctypes.data, len(q_rows), dq.ctypes.data,
+                                 k_rows.ctypes.data, len(k_rows), dk.ctypes.data, dv.ctypes.data)
+    if rc != 0:
+        raise ValueError("ksa_oracle_bwd_rows: bad arguments (%d)" % rc)
     return dq, dk, dv

@@ -54,7 +54,7 @@ constexpr int kRegsOther = 72;
 static_assert(8 * kRegsSoftmax + 4 * kRegsOther <= 12 * ((65536 / kThreads) / 8 * 8), "register hand-over exceeds the CTA's allocation");
 constexpr int kQkWarp = 11, kPvWarp = 9, kKProdWarp = 8, kVProdWarp = 10;
 #ifndef KSA_RESCALE_T
-#define KSA_RESCALE_T 12.0f
+#define KSA_RESCALE_T 8.0f
 #endif
 constexpr float kRescaleThreshold = KSA_RESCALE_T;
 constexpr int D = 128;

@@ -137,3 +137,34 @@ def test_row_costs_add_up_to_the_oracle_pair_count():
         for a in (0, 1, L // 2, L - 1):
             assert dist_utils.visible_pairs_of_rows(n, k, m, C, a, a + 1) == orc.visible_count(n, k, m, C, a)
         assert dist_utils.visible_pairs_of_rows(n, k, m, C, 0, L) == dist_utils.visible_pairs_of_sequence(n, k, m, C)
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` outside torchrun starts two ranks of itself (here with the stand-in step over gloo: no
+    GPU in this test), the slower rank sets the time and rank 0 alone prints one line with n_gpus = 2."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    env["KSA_BENCH_LAUNCH_TEST"] = "1"
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "5", "--warmup", "1"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    assert lines[0]["n_gpus"] == 2 and lines[0]["built_by_launcher"]
+    assert lines[0]["ms_per_step"] >= 2.0           # rank 1 sleeps 2 ms per step: the MAX over ranks
+
+
+def test_bench_gpus_flag_fails_loudly_without_enough_gpus():
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "KSA_BENCH_LAUNCH_TEST")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "64", "--steps", "1"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode != 0
+    assert "GPU" in (r.stderr + r.stdout) or "CUDA" in (r.stderr + r.stdout)

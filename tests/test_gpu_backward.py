@@ -127,6 +127,87 @@ def test_backward_full_size_identities(ctx, workload):
     assert (qabs > 0).all() and (vabs > 0).all()
 
 
+def _aug_of_text(n, k, m, i):
+    J = n // k
+    return (i // k) * (k + m) + i % k if i < J * k else J * (k + m) + (i - J * k)
+
+
+def _check_rows(name, got, ref):
+    """Sampled rows: the same bounds as _check, with each tensor's scale taken from the sample."""
+    assert np.isfinite(got).all(), name
+    err = np.abs(got - ref)
+    assert err.max() <= 2e-2 * np.abs(ref).max() + 1e-5, (name, err.max(), np.abs(ref).max())
+    assert err.mean() <= 1e-2 * np.abs(ref).mean() + 1e-5, (name, err.mean(), np.abs(ref).mean())
+    # row by row as well: a row that is wrong as a whole must not hide behind the sample's largest row
+    rerr = err.reshape(err.shape[0], -1).max(axis=1)
+    rref = np.abs(ref).reshape(ref.shape[0], -1).max(axis=1)
+    assert (rerr <= 4e-2 * rref + 2e-2 * np.abs(ref).max() * 0.05 + 1e-5).all(), (name, rerr, rref)
+
+
+@pytest.mark.parametrize("workload", ["32k", "128k", "varlen"])
+def test_backward_full_size_sampled_rows(ctx, workload):
+    """Full-size workloads in the launch configuration the bench times, element by element on sampled rows against
+    the oracle's fp64 gradients (ksa_oracle_bwd_rows: dq of a row needs that row only; dk, dv of a key need every
+    query row that sees it under Eq. 3, each with its complete softmax).
+
+    Query rows: first and last rows, rows either side of tile and window boundaries, summary rows, random rows.
+    Key rows: text keys (first, last, tile edges, random) -- each is seen by the window's ~1,032 query rows, i.e. by
+    nine query tiles -- and summary keys.  At 32k a summary key of the first chunks is sampled, which every later
+    row sees: 256 query tiles, sixteen accumulation segments of the dK/dV kernel, four query heads per KV head.
+    At 128k and in the long sequences of varlen the sampled summary keys are late ones (seen by the last few
+    thousand rows: two segments), because the oracle needs the complete softmax of every row that sees a sampled
+    key; there the early keys stay covered by the sum identities of the test above."""
+    wl = synth.WORKLOADS[workload]
+    lay = synth.LAYOUT_P
+    k, m, C = lay.k, lay.m, lay.C
+    dev = torch.device("cuda", 0)
+    prob = ksa.Problem(wl.text_lens, k, m, C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    total = ksa.total_aug_len(prob)
+    q, kk, v = synth.make_qkv(wl, total)
+    qd, kd, vd = q.to(dev), kk.to(dev), v.to(dev)
+    g = torch.Generator("cpu").manual_seed(5)
+    dout = torch.randn((total, wl.Hq, wl.D), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    gd = dout.to(dev)
+    out = torch.empty_like(qd); lse = torch.empty((wl.Hq, total), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx.clear_device_status()
+    ctx.attn_fwd(prob, qd, kd, vd, out, lse, ws)
+    dq = torch.full_like(qd, 7.0); dk = torch.full_like(kd, 7.0); dv = torch.full_like(vd, 7.0)
+    wsb = torch.full((ksa.bwd_workspace_bytes(prob),), 0xFF, dtype=torch.uint8, device=dev)
+    ctx.attn_bwd(prob, qd, kd, vd, out, lse, gd, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+
+    rng = np.random.default_rng(17)
+    q_rows, k_rows = [], []
+    base = 0
+    lens = list(wl.text_lens)
+    # which sequences get key samples: all at 32k, the one sequence at 128k, the shortest and the longest of varlen
+    key_seqs = set(range(len(lens))) if len(lens) <= 2 else {int(np.argmin(lens)), int(np.argmax(lens))}
+    for b, n in enumerate(lens):
+        L = orc.aug_len(n, k, m)
+        J = n // k
+        text = [0, 1, 127, 128, C * k - 1, C * k + k, n // 2, n - 129, n - 2, n - 1] + [int(t) for t in rng.integers(0, n, size=4)]
+        text = sorted(set(min(max(t, 0), n - 1) for t in text))
+        q_rows += [base + _aug_of_text(n, k, m, t) for t in text]
+        q_rows += [base + j * (k + m) + k for j in (0, J // 2, J - 1)]              # summary rows
+        if b in key_seqs:
+            tk = [0, 127, 128, n - 1, n - 130] + [int(t) for t in rng.integers(0, n, size=3)]
+            k_rows += [base + _aug_of_text(n, k, m, min(max(t, 0), n - 1)) for t in sorted(set(tk))]
+            late = [J - 1, J - C - 2, J - C - 2 - 200]                                # seen by nobody / few / ~1,600 text rows
+            early = [1] if n <= 40000 else []                                        # seen by nearly every row
+            k_rows += [base + j * (k + m) + k for j in late + early if 0 <= j < J]
+        base += L
+    q_rows = np.unique(np.asarray(q_rows, dtype=np.int64))
+    k_rows = np.unique(np.asarray(k_rows, dtype=np.int64))
+    rdq, rdk, rdv = orc.bwd_rows(synth.bits(q), synth.bits(kk), synth.bits(v), synth.bits(dout), lens, k, m, C, wl.scale,
+                                 q_rows, k_rows)
+    tq = torch.from_numpy(q_rows).to(dev); tk_ = torch.from_numpy(k_rows).to(dev)
+    _check_rows("dq", dq[tq].double().cpu().numpy(), rdq)
+    _check_rows("dk", dk[tk_].double().cpu().numpy(), rdk)
+    _check_rows("dv", dv[tk_].double().cpu().numpy(), rdv)
+
+
 def test_full_causal_mode_against_torch_attention(ctx):
     """m = 0 and a window that covers every chunk reduce the operator to plain causal attention: forward and
     backward against torch's scaled_dot_product_attention and autograd in fp32 on the same bf16 inputs (a library

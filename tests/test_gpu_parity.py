@@ -58,9 +58,20 @@ def test_full_size_sampled(ctx, name, n_random):
     parity.check_workload(ctx, synth.WORKLOADS[name], synth.LAYOUT_P, 0, n_random=n_random, seed=11)
 
 
-def test_full_size_layout_g_sampled(ctx):
-    """128K at the 64 + 8 chunk layout (m = 8 summaries per chunk), sampled rows."""
-    parity.check_workload(ctx, synth.WORKLOADS["128k"], synth.LAYOUT_G, 0, n_random=256, seed=12)
+@pytest.mark.parametrize("name,n_random", [("32k", 384), ("128k", 256), ("varlen", 512)])
+def test_full_size_layout_g_sampled(ctx, name, n_random):
+    """The large workloads at the 64 + 8 chunk layout (m = 8 summaries per chunk), sampled rows (boundary tiles of every
+    sequence plus random rows)."""
+    parity.check_workload(ctx, synth.WORKLOADS[name], synth.LAYOUT_G, 0, n_random=n_random, seed=12)
+
+
+@pytest.mark.parametrize("name,layout,n_random", [("8k", "P", 0), ("32k", "P", 384), ("128k", "P", 256), ("varlen", "P", 384),
+                                                  ("32k", "G", 256), ("128k", "G", 192)])
+def test_cta_pair_kernel(ctx, name, layout, n_random):
+    """The CTA-pair text kernel (opt-in flag) on the workloads it applies to, against the oracle; the ragged varlen
+    batch goes through the packed streams, the others are read in place."""
+    lay = {"P": synth.LAYOUT_P, "G": synth.LAYOUT_G}[layout]
+    parity.check_workload(ctx, synth.WORKLOADS[name], lay, ksa.KSA_FLAG_CTA_PAIR_KERNEL, n_random=n_random, seed=13)
 
 
 @pytest.mark.parametrize("kernel_flag", [REF, 0], ids=["ref", "tc"])
@@ -82,6 +93,20 @@ def test_full_size_layout_g_sampled(ctx):
 def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
     wl = synth.Workload("edge", 99, lens, Hq, Hkv, D)
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), kernel_flag)
+
+
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv", [
+    ([1], 8, 1, 2, 2, 1), ([7], 8, 1, 2, 2, 1), ([127, 129, 128], 8, 1, 3, 4, 2), ([333, 1000], 3, 2, 5, 4, 2),
+    ([777], 16, 0, 7, 4, 2), ([640], 1, 1, 100, 2, 1), ([1290], 200, 3, 1, 4, 1), ([2048, 640, 1336], 8, 1, 16, 8, 2),
+    ([768], 128, 1, 2, 2, 1), ([2100], 8, 1, 16, 8, 2), ([4096], 64, 8, 4, 4, 2), ([130], 8, 1, 0, 16, 2),
+])
+@pytest.mark.parametrize("strict", [0, STRICT])
+def test_cta_pair_kernel_edge_shapes(ctx, lens, k, m, C, Hq, Hkv, strict):
+    """Edge shapes through the CTA-pair kernel (head_dim 128, even group sizes): single tokens, ragged tiles, chunks that do
+    not divide a tile (falls back to packed streams), no summaries, items of one and two tiles (the tile stream runs
+    across work items), more work items than pairs and fewer."""
+    wl = synth.Workload("pair-edge", 98, lens, Hq, Hkv, 128)
+    parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), ksa.KSA_FLAG_CTA_PAIR_KERNEL | strict)
 
 
 @pytest.mark.parametrize("n", [900, 896])     # 896: whole chunks, tiles are read straight from the strided views

@@ -108,3 +108,31 @@ def test_gradient_identities():
     qb3[Ls[0]:] ^= 0x0101; kb3[Ls[0]:] ^= 0x0101; vb3[Ls[0]:] ^= 0x0101
     dq3, dk3, dv3 = orc.bwd(qb3, kb3, vb3, gb, lens, k, m, C, scale)
     assert np.array_equal(dq3[:Ls[0]], dq[:Ls[0]]) and np.array_equal(dk3[:Ls[0]], dk[:Ls[0]]) and np.array_equal(dv3[:Ls[0]], dv[:Ls[0]])
+
+
+def test_sampled_rows_equal_the_full_gradients():
+    """ksa_oracle_bwd_rows (the gradients of a sample of rows, used where the full computation is too long) returns
+    exactly the corresponding rows of ksa_oracle_bwd, whose arithmetic the tests above pin: packed sequences, GQA,
+    ragged tail, keys that are text and keys that are summaries, rows in every sequence."""
+    rng = np.random.default_rng(3)
+    lens, k, m, C, Hq, Hkv, D = [70, 33, 9], 4, 2, 3, 4, 2, 8
+    total = sum(orc.aug_len(n, k, m) for n in lens)
+    rand_bf16 = helpers.rand_bf16
+    qb, _ = rand_bf16(rng, (total, Hq, D))
+    kb, _ = rand_bf16(rng, (total, Hkv, D))
+    vb, _ = rand_bf16(rng, (total, Hkv, D))
+    gb, _ = rand_bf16(rng, (total, Hq, D))
+    dq, dk, dv = orc.bwd(qb, kb, vb, gb, lens, k, m, C, 0.35)
+    q_rows = np.array([0, 3, 5, 17, 60, total - 1, orc.aug_len(70, k, m), orc.aug_len(70, k, m) + 20], dtype=np.int64)
+    k_rows = np.array([0, 4, 5, 11, 40, 104, 105 + 7, total - 2], dtype=np.int64)     # rows 4, 5, 11: summaries of sequence 0
+    sq, sk, sv = orc.bwd_rows(qb, kb, vb, gb, lens, k, m, C, 0.35, q_rows, k_rows)
+    np.testing.assert_allclose(sq, dq[q_rows], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(sk, dk[k_rows], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(sv, dv[k_rows], rtol=1e-12, atol=1e-14)
+    assert np.abs(sk).max() > 0 and np.abs(sq).max() > 0
+    # the strict summary rule goes through the same predicate
+    dq2, dk2, dv2 = orc.bwd(qb, kb, vb, gb, lens, k, m, C, 0.35, orc.SUMMARY_TEXT_ONLY)
+    sq2, sk2, sv2 = orc.bwd_rows(qb, kb, vb, gb, lens, k, m, C, 0.35, q_rows, k_rows, orc.SUMMARY_TEXT_ONLY)
+    np.testing.assert_allclose(sq2, dq2[q_rows], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(sk2, dk2[k_rows], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(sv2, dv2[k_rows], rtol=1e-12, atol=1e-14)
