@@ -55,6 +55,7 @@ extern "C" {
 #define KSA_ERR_CUDA          -4   /* a CUDA runtime/driver call failed (see ksa_last_cuda_error)      */
 #define KSA_ERR_TIMEOUT       -5   /* a bounded device-side wait gave up (see ksa_last_device_status)  */
 #define KSA_ERR_NOMEM         -6   /* host allocation failed                                           */
+#define KSA_ERR_INTERNAL      -7   /* the library's own schedule failed its range check: nothing was launched */
 
 /* ---- flags -------------------------------------------------------------------------- */
 /* Summary rows see the text of their own chunk only (strict reading of Sec. 2.2.1).

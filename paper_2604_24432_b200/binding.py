@@ -15,11 +15,12 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libksa_b200.so")
+# KSA_B200_LIB_VARIANT=debug / asan selects a test variant of the library (see build.py); unset: the product library
+LIB_PATH = os.path.join(_HERE, "libksa_b200%s.so" % ("_" + os.environ["KSA_B200_LIB_VARIANT"] if os.environ.get("KSA_B200_LIB_VARIANT") else ""))
 
 KSA_OK = 0
 KSA_ERR_INVALID_ARG, KSA_ERR_UNSUPPORTED, KSA_ERR_WORKSPACE = -1, -2, -3
-KSA_ERR_CUDA, KSA_ERR_TIMEOUT, KSA_ERR_NOMEM = -4, -5, -6
+KSA_ERR_CUDA, KSA_ERR_TIMEOUT, KSA_ERR_NOMEM, KSA_ERR_INTERNAL = -4, -5, -6, -7
 KSA_PREP_NO_ROPE = 1
 KSA_FLAG_SUMMARY_TEXT_ONLY = 0x1
 KSA_FLAG_REFERENCE_KERNEL = 0x2

@@ -276,6 +276,33 @@ void build_schedule(const ksa_params* p, HostSchedule& hs, int target_chunks)
     }
 }
 
+// Range check of a freshly built schedule, before it is ever uploaded: every field a kernel will index with.
+static bool schedule_in_range(const ksa_params* p, const HostSchedule& hs)
+{
+    const int G = p->num_q_heads / p->num_kv_heads;
+    int64_t aug = 0;
+    for (const SeqInfo& s : hs.seqs) {
+        if (s.aug_off != aug || s.n_text < 1 || s.text_pad % kTileM || s.summ_pad % kTileN) return false;
+        if (s.text_off < 0 || s.text_off + (int64_t)s.text_pad > hs.text_rows) return false;
+        if (s.summ_off < 0 || s.summ_off + (int64_t)s.summ_pad > hs.summ_rows) return false;
+        aug += (int64_t)s.n_text + s.n_summ;
+    }
+    if (aug != hs.total_aug) return false;
+    for (const WorkItem& w : hs.work) {
+        if (w.seq < 0 || w.seq >= (int)hs.seqs.size()) return false;
+        const SeqInfo& s = hs.seqs[w.seq];
+        if (w.q_tile < 0 || (int64_t)w.q_tile * kTileM >= s.text_pad) return false;
+        if (w.n_heads < 1 || w.n_heads > 2 || w.head0 < 0 || w.head0 + w.n_heads > p->num_q_heads) return false;
+        if (w.head0 / G != (w.head0 + w.n_heads - 1) / G) return false;                     // one KV head per item
+        if (w.ns_tiles < 0 || (int64_t)w.ns_tiles * kTileN > s.summ_pad || w.ns_nomask < 0 || w.ns_nomask > w.ns_tiles) return false;
+        if (w.band_lo < 0 || w.band_hi < w.band_lo || w.band_hi != w.q_tile) return false;
+        if (w.band_nomask_lo < w.band_lo || w.band_nomask_hi > w.band_hi + 1 || w.band_nomask_hi < w.band_nomask_lo) return false;
+    }
+    for (const RowChunk& c : hs.chunks)
+        if (c.work_off < 0 || c.work_off + c.work_cnt > (int64_t)hs.work.size() || c.aug0 < 0 || c.aug1 > hs.total_aug || c.aug1 < c.aug0) return false;
+    return true;
+}
+
 static std::vector<int32_t> schedule_key(const ksa_params* p)
 {
     std::vector<int32_t> key;
@@ -367,6 +394,7 @@ extern "C" __attribute__((visibility("default"))) const char* ksa_strerror(int s
         case KSA_ERR_CUDA: return "CUDA call failed";
         case KSA_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case KSA_ERR_NOMEM: return "out of host memory";
+        case KSA_ERR_INTERNAL: return "the library's schedule failed its own range check";
         default: return "unknown status";
     }
 }
@@ -482,6 +510,7 @@ static int ensure_schedule(ksa_ctx* ctx, const ksa_params* p, bool upload, int t
             build_layout(p, hs);
             build_schedule(p, hs, target_chunks);
         } catch (const std::bad_alloc&) { return KSA_ERR_NOMEM; }
+        if (!schedule_in_range(p, hs)) return KSA_ERR_INTERNAL;
         hs.key = key;
         ctx->sched = std::move(hs);
         // the device copies belong to the old schedule (cudaFree waits for work in flight)

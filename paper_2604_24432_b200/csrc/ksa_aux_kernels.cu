@@ -75,6 +75,10 @@ __global__ void __launch_bounds__(256) ksa_pack_kernel(KernelArgs a)
             }
         }
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        // (debug builds) the source row inside the caller's tensors, the destination row inside its stream
+        const bool in_range = ksa_in_bounds(aug >= 0 && aug < a.total_aug && row >= 0 &&
+                                            (int64_t)(text ? sq.text_off : sq.summ_off) + row < (text ? a.text_rows : a.summ_rows), a.status);
+        if (!in_range) continue;
         if (row < live_rows) val = *reinterpret_cast<const uint4*>(src + vec * 8);
         *reinterpret_cast<uint4*>(dst + vec * 8) = val;
     }
@@ -204,7 +208,7 @@ __device__ __forceinline__ void summ_long_tasks(const KernelArgs& a, const uint1
                 }
             }
         }
-        if (live) {
+        if (live && ksa_out_row_ok(a, qrow, h)) {
             const float inv = 1.f / l;
             uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * E;
 #pragma unroll
@@ -408,7 +412,7 @@ __global__ void __launch_bounds__(256) ksa_summary_short_kernel(KernelArgs a)
                 }
             }
         }
-        if (live) {
+        if (live && ksa_out_row_ok(a, qrow, h)) {
             const float inv = 1.f / l;
             uint16_t* op = a.out + qrow * a.o_st + (int64_t)h * a.o_sh + sub * 8;
 #pragma unroll
@@ -519,10 +523,12 @@ __global__ void __launch_bounds__(256) ksa_text_ref_kernel(KernelArgs a)
         }
         const float inv = 1.f / l;
         const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * s + (i % a.k);
-        uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
+        if (ksa_out_row_ok(a, aug, h)) {
+            uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
 #pragma unroll
-        for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
-        if (lane == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
+            for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
+            if (lane == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
+        }
     }
 }
 

@@ -78,6 +78,26 @@ enum DeviceStatus : int32_t {
     kStatusWaitRowSums = 11,    // CTA-pair kernel: the other softmax group's row sums
     kStatusWaitPvDone = 12,     // CTA-pair kernel: completion of O += P V
     kStatusWaitOEmpty = 13,     // CTA-pair kernel: the epilogue's read of O
+    kStatusBounds = 14,         // KSA_DEBUG builds: a global output index was outside its tensor; the access was skipped
 };
+
+// KSA_DEBUG builds (the stand-in for a memory checker): every global store of the kernels goes through ksa_in_bounds,
+// which records kStatusBounds and makes the caller skip the access when the index is outside the tensor.
+#if defined(__CUDACC__)
+#ifdef KSA_DEBUG
+__device__ __forceinline__ bool ksa_in_bounds(bool ok, int32_t* status)
+{
+    if (!ok) atomicCAS(status, 0, (int32_t)kStatusBounds);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool ksa_in_bounds(bool, int32_t*) { return true; }
+#endif
+// a row of out (and its lse entry) addressed by augmented row and query head
+__device__ __forceinline__ bool ksa_out_row_ok(const KernelArgs& a, int64_t aug, int h)
+{
+    return ksa_in_bounds(aug >= 0 && aug < a.total_aug && h >= 0 && h < a.Hq, a.status);
+}
+#endif
 
 }  // namespace ksa

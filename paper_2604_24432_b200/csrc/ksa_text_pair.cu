@@ -734,12 +734,13 @@ ksa_text_pair_kernel(const __grid_constant__ KernelArgs a, const __grid_constant
             const int h = w.head0 + (int)rank;
             const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * s_len + (i % a.k);
             uint16_t* orow = a.out + aug * a.o_st + (int64_t)h * a.o_sh + wg * 64;
+            const bool store = valid && ksa_out_row_ok(a, aug, h);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tO + wg * 64 + c * 32, o);
                 tc_wait_ld();
-                if (valid) {
+                if (store) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint4 pk;
@@ -751,7 +752,7 @@ ksa_text_pair_kernel(const __grid_constant__ KernelArgs a, const __grid_constant
                     }
                 }
             }
-            if (valid && wg == 0) a.lse[(int64_t)h * a.total_aug + aug] = (m_fin + log2f(l_tot)) * 0.6931471805599453f;
+            if (store && wg == 0) a.lse[(int64_t)h * a.total_aug + aug] = (m_fin + log2f(l_tot)) * 0.6931471805599453f;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster_relaxed(lead(bar(B_OEMPTY)));

@@ -442,12 +442,13 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             const int h = w.head0 + t;
             const int64_t aug = sq.aug_off + (int64_t)(i / a.k) * s_len + (i % a.k);
             uint16_t* orow = a.out + aug * a.o_st + (int64_t)h * a.o_sh;
+            const bool store = valid && ksa_out_row_ok(a, aug, h);
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tO + c * 32, o);
                 tc_wait_ld();
-                if (valid) {
+                if (store) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint4 pk;
@@ -459,7 +460,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     }
                 }
             }
-            if (valid) a.lse[(int64_t)h * a.total_aug + aug] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+            if (store) a.lse[(int64_t)h * a.total_aug + aug] = (m_used + log2f(l_run)) * 0.6931471805599453f;
             tc_fence_before();
         }
     }
