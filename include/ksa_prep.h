@@ -47,6 +47,25 @@ int ksa_qkv_prepare(ksa_ctx* ctx, const void* q_main, const void* k_main, const 
                     void* q_out, void* k_out, void* v_out, float lambda, float rope_theta, uint32_t prep_flags,
                     const ksa_params* p, void* cuda_stream);
 
+/*
+ * Preparation and attention in one call, with the preparation folded into the pass that de-interleaves
+ * q, k, v for the attention kernels: the projections are read once, position ids (Sec. 2.2.1), interpolation
+ * at summary positions (Sec. 4.1) and rotation are applied on the way, and the prepared rows are written
+ * straight into the packed streams the tensor-core kernel reads -- no prepared copy of q, k, v is ever
+ * stored in the interleaved layout, and the whole step moves q, k and v through HBM once in and once out
+ * (what ksa_qkv_prepare alone costs).  Works for any lengths; results equal
+ * ksa_qkv_prepare followed by ksa_attn_fwd bit for bit (same arithmetic on the same rows).
+ * q_main .. v_summ, lambda, rope_theta, prep_flags: as for ksa_qkv_prepare; out, lse, p, cuda_stream: as for
+ * ksa_attn_fwd (KSA_FLAG_REFERENCE_KERNEL is not accepted).  workspace: DEVICE, 256-byte aligned,
+ * >= ksa_prepared_workspace_bytes (the packed streams plus the prepared query rows of the summary tokens).
+ */
+int ksa_prepared_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
+int ksa_attn_fwd_prepared(ksa_ctx* ctx, const void* q_main, const void* k_main, const void* v_main,
+                          const void* q_summ, const void* k_summ, const void* v_summ,
+                          float lambda, float rope_theta, uint32_t prep_flags,
+                          void* out, float* lse, void* workspace, size_t workspace_bytes,
+                          const ksa_params* p, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,6 +38,7 @@ EXPORTS = [
     "ksa_cache_rows", "ksa_cache_bytes", "ksa_cache_slice", "ksa_cache_reset", "ksa_cache_fill_from_prefill",
     "ksa_decode_text", "ksa_decode_summary",
     "ksa_anneal_lambda", "ksa_position_ids", "ksa_total_summary_rows", "ksa_qkv_prepare",
+    "ksa_prepared_workspace_bytes", "ksa_attn_fwd_prepared",
     "ksa_part_rows", "ksa_attn_fwd_part",
 ]
 
@@ -115,6 +116,8 @@ def lib():
     L.ksa_total_summary_rows.restype = i64
     L.ksa_total_summary_rows.argtypes = [pp]
     L.ksa_qkv_prepare.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, pp, vp]
+    L.ksa_prepared_workspace_bytes.argtypes = [vp, pp, ctypes.POINTER(ctypes.c_size_t)]
+    L.ksa_attn_fwd_prepared.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp, vp, ctypes.c_size_t, pp, vp]
     L.ksa_schedule_dump.argtypes = [vp, pp, ctypes.POINTER(ksa_tile_rec), i64, ctypes.POINTER(i64)]
     L.ksa_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.ksa_selftest_bounded_wait.argtypes = [vp, i64, vp, vp]
@@ -219,6 +222,13 @@ def anneal_lambda(step: int, s_start: int, s_end: int) -> float:
     lam = ctypes.c_float()
     _check(lib().ksa_anneal_lambda(step, s_start, s_end, ctypes.byref(lam)), "ksa_anneal_lambda")
     return float(lam.value)
+
+
+def prepared_workspace_bytes(prob: Problem) -> int:
+    b = ctypes.c_size_t()
+    p = prob.params()
+    _check(lib().ksa_prepared_workspace_bytes(None, ctypes.byref(p), ctypes.byref(b)), "ksa_prepared_workspace_bytes")
+    return int(b.value)
 
 
 def position_ids(prob: Problem):
@@ -334,6 +344,20 @@ class Context:
                                      ptr(q_summ), ptr(k_summ), ptr(v_summ), q_out.data_ptr(), k_out.data_ptr(), v_out.data_ptr(),
                                      ctypes.c_float(lam), ctypes.c_float(rope_theta), ctypes.c_uint32(flags),
                                      ctypes.byref(p), stream), "ksa_qkv_prepare")
+
+    def attn_fwd_prepared(self, prob: Problem, q_main, k_main, v_main, q_summ, k_summ, v_summ, lam: float, rope_theta: float,
+                          out, lse, workspace, flags: int = 0, stream: Optional[int] = None):
+        """ksa_attn_fwd_prepared: preparation (position ids, interpolation, rotation) folded into the pack pass, then attention."""
+        import torch
+        p = prob.params(q_main, k_main, v_main, out)
+        if stream is None:
+            stream = torch.cuda.current_stream(q_main.device).cuda_stream
+        ptr = lambda t: None if t is None else t.data_ptr()
+        _check(lib().ksa_attn_fwd_prepared(self.handle, q_main.data_ptr(), k_main.data_ptr(), v_main.data_ptr(),
+                                           ptr(q_summ), ptr(k_summ), ptr(v_summ), ctypes.c_float(lam), ctypes.c_float(rope_theta),
+                                           ctypes.c_uint32(flags), out.data_ptr(), lse.data_ptr(), workspace.data_ptr(),
+                                           workspace.numel() * workspace.element_size(), ctypes.byref(p), stream),
+               "ksa_attn_fwd_prepared")
 
     def attn_fwd_host(self, prob: Problem, q, k, v, out, lse, staging, stream: Optional[int] = None):
         """ksa_attn_fwd_host: q, k, v, out, lse are contiguous HOST tensors (pinned recommended)."""

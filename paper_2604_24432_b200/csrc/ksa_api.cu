@@ -1052,6 +1052,88 @@ extern "C" __attribute__((visibility("default"))) int ksa_qkv_prepare(ksa_ctx* c
     return KSA_OK;
 }
 
+// ---- preparation fused into the pack pass (include/ksa_prep.h) ------------------------------------------
+// Workspace: the five packed streams of the forward pass, then the prepared query rows of the summary tokens.
+static size_t prepared_ws_bytes(const ksa_params* p, const HostSchedule& hs, size_t* qs_off)
+{
+    const WorkspaceLayout wl = workspace_layout(p, hs);
+    if (qs_off) *qs_off = wl.total;
+    return wl.total + (size_t)round_up((int64_t)((size_t)p->num_q_heads * hs.summ_rows * p->head_dim * 2), 1024);
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_prepared_workspace_bytes(const ksa_ctx*, const ksa_params* p, size_t* bytes)
+{
+    if (!bytes) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    HostSchedule hs;
+    build_layout(p, hs);
+    *bytes = prepared_ws_bytes(p, hs, nullptr);
+    return KSA_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int ksa_attn_fwd_prepared(ksa_ctx* ctx, const void* q_main, const void* k_main, const void* v_main,
+                                     const void* q_summ, const void* k_summ, const void* v_summ,
+                                     float lambda, float rope_theta, uint32_t prep_flags,
+                                     void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                     const ksa_params* p, void* cuda_stream)
+{
+    if (!ctx || !q_main || !k_main || !v_main || !out || !lse) return KSA_ERR_INVALID_ARG;
+    int rc = validate(p);
+    if (rc != KSA_OK) return rc;
+    if ((rc = validate_strides(p)) != KSA_OK) return rc;
+    if (p->flags & KSA_FLAG_REFERENCE_KERNEL) return KSA_ERR_INVALID_ARG;
+    if (!(lambda >= 0.f && lambda <= 1.f)) return KSA_ERR_INVALID_ARG;
+    const bool rope = !(prep_flags & KSA_PREP_NO_ROPE);
+    if (rope && !(rope_theta > 0.f)) return KSA_ERR_INVALID_ARG;
+    const bool need_summ = lambda != 0.f && ksa_total_summary_rows(p) > 0;
+    if (need_summ && (!q_summ || !k_summ || !v_summ)) return KSA_ERR_INVALID_ARG;
+    const uintptr_t ptrs[8] = {(uintptr_t)q_main, (uintptr_t)k_main, (uintptr_t)v_main, (uintptr_t)q_summ, (uintptr_t)k_summ,
+                               (uintptr_t)v_summ, (uintptr_t)out, (uintptr_t)lse};
+    for (int i = 0; i < 8; ++i) if (ptrs[i] & 15) return KSA_ERR_INVALID_ARG;
+    if ((rc = ensure_schedule(ctx, p, true)) != KSA_OK) return rc;
+    const HostSchedule& hs = ctx->sched;
+    size_t qs_off = 0;
+    const size_t need = prepared_ws_bytes(p, hs, &qs_off);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return KSA_ERR_WORKSPACE;
+    const WorkspaceLayout wl = workspace_layout(p, hs);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // the attention kernels read the packed streams only (a.direct = 0); q, k, v of the arguments are the projections
+    KernelArgs a = make_args(ctx, p, q_main, k_main, v_main, out, lse, workspace, wl, false);
+    uint16_t* qs = (uint16_t*)((char*)workspace + qs_off);
+
+    PrepArgs pa{};
+    pa.seqs = ctx->d_seqs;
+    pa.k = p->chunk_len; pa.m = p->summaries_per_chunk; pa.Hq = p->num_q_heads; pa.Hkv = p->num_kv_heads; pa.D = p->head_dim;
+    pa.rope = rope ? 1 : 0;
+    pa.lambda = need_summ ? lambda : 0.f;
+    for (int d = 0; d < p->head_dim / 2 && d < 64; ++d)
+        pa.inv_freq[d] = rope ? std::pow((double)rope_theta, -2.0 * d / (double)p->head_dim) : 0.0;
+    pa.qm = (const uint16_t*)q_main; pa.km = (const uint16_t*)k_main; pa.vm = (const uint16_t*)v_main;
+    pa.qs = (const uint16_t*)q_summ; pa.ks = (const uint16_t*)k_summ; pa.vs = (const uint16_t*)v_summ;
+    pa.q_st = p->q_stride_tok; pa.q_sh = p->q_stride_head; pa.k_st = p->k_stride_tok; pa.k_sh = p->k_stride_head;
+    pa.v_st = p->v_stride_tok; pa.v_sh = p->v_stride_head;
+    pa.to_streams = 1;
+    pa.qt = a.qt; pa.kt = a.kt; pa.vt = a.vt; pa.ks_out = a.ks; pa.vs_out = a.vs; pa.qs_out = qs;
+    pa.text_rows = hs.text_rows; pa.summ_rows = hs.summ_rows;
+    int64_t max_aug_len = 0;
+    for (const SeqInfo& sq : hs.seqs) max_aug_len = std::max<int64_t>(max_aug_len, (int64_t)sq.n_text + sq.n_summ);
+    cudaError_t e;
+    if ((e = launch_zero_stream_pads(pa, p->num_seqs, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = launch_prep(pa, max_aug_len, p->num_seqs, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 2;
+    if (a.m > 0 && a.max_n_summ > 0) {
+        if ((e = launch_summary_streams(a, qs, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
+    if (ctx->timing) cudaEventRecord(ctx->ev0, stream);
+    FwdMaps maps;
+    if ((rc = prepare_text(ctx, a, p->flags, maps)) != KSA_OK) return rc;
+    if ((rc = launch_text(ctx, a, p->flags, maps, stream)) != KSA_OK) return rc;
+    if (ctx->timing) { cudaEventRecord(ctx->ev1, stream); ctx->timing_valid = true; }
+    return KSA_OK;
+}
+
 struct StagingLayout { size_t q, k, v, out, lse, ws, ws_bytes, total; };
 static int staging_layout(const ksa_params* p, StagingLayout& s)
 {

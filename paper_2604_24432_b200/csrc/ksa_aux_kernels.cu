@@ -532,6 +532,72 @@ __global__ void __launch_bounds__(256) ksa_text_ref_kernel(KernelArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Summary rows from the packed streams (the path whose preparation pass wrote the streams directly, so that no
+// prepared interleaved tensors exist): one warp per (summary row, query head); lane l holds D / 32 elements.
+// Keys of summary (j, r): text rows [j k, j k + k) of the text stream, then summary rows j m .. j m + r of the
+// summary stream (Sec. 2.2.1; the latter not under KSA_FLAG_SUMMARY_TEXT_ONLY).  One key at a time, online softmax.
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) ksa_summary_streams_kernel(KernelArgs a, const uint16_t* __restrict__ qs)
+{
+    constexpr int E = D / 32;
+    const SeqInfo sq = a.seqs[blockIdx.y];
+    const int lane = threadIdx.x & 31;
+    const int G = a.Hq / a.Hkv;
+    const int64_t tasks = (int64_t)sq.n_summ * a.Hq;
+    for (int64_t task = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); task < tasks; task += (int64_t)gridDim.x * 8) {
+        const int u = (int)(task / a.Hq), h = (int)(task % a.Hq), hk = h / G;
+        const int j = u / a.m, r = u % a.m;
+        float qv[E];
+        const uint16_t* qp = qs + ((int64_t)h * a.summ_rows + sq.summ_off + u) * D + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) qv[e] = __uint_as_float((uint32_t)qp[e] << 16);
+        float mx = -INFINITY, l = 0.f, acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        const int n_summ_keys = (a.flags & 0x1u) ? 0 : r + 1;
+        for (int t = 0; t < a.k + n_summ_keys; ++t) {
+            const bool text = t < a.k;
+            const int64_t row = text ? (int64_t)sq.text_off + (int64_t)j * a.k + t : (int64_t)sq.summ_off + (int64_t)j * a.m + (t - a.k);
+            const int64_t off = ((int64_t)hk * (text ? a.text_rows : a.summ_rows) + row) * D + lane * E;
+            const uint16_t* kp = (text ? a.kt : a.ks) + off;
+            const uint16_t* vp = (text ? a.vt : a.vs) + off;
+            float dot = 0.f;
+#pragma unroll
+            for (int e = 0; e < E; ++e) dot = fmaf(qv[e], __uint_as_float((uint32_t)kp[e] << 16), dot);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            const float sc = dot * a.scale;
+            const float m_new = fmaxf(mx, sc);
+            const float corr = __expf(mx - m_new), p = __expf(sc - m_new);
+            l = l * corr + p;
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] = fmaf(p, __uint_as_float((uint32_t)vp[e] << 16), acc[e] * corr);
+            mx = m_new;
+        }
+        const int64_t aug = sq.aug_off + (int64_t)j * (a.k + a.m) + a.k + r;
+        if (ksa_out_row_ok(a, aug, h)) {
+            const float inv = 1.f / l;
+            uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
+#pragma unroll
+            for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
+            if (lane == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
+        }
+    }
+}
+
+cudaError_t launch_summary_streams(const KernelArgs& a, const uint16_t* qs, cudaStream_t stream)
+{
+    if (a.m <= 0 || a.max_n_summ <= 0) return cudaSuccess;
+    int64_t blocks = ((int64_t)a.max_n_summ * a.Hq + 7) / 8;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, 1u);
+    if (a.D == 128) ksa_summary_streams_kernel<128><<<grid, 256, 0, stream>>>(a, qs);
+    else            ksa_summary_streams_kernel<64><<<grid, 256, 0, stream>>>(a, qs);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_text_ref(const KernelArgs& a, cudaStream_t stream)
 {
     if (a.num_work <= 0) return cudaSuccess;

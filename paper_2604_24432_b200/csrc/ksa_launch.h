@@ -46,7 +46,18 @@ struct PrepArgs {
     const uint16_t* qs; const uint16_t* ks; const uint16_t* vs;     // ... with the summary weights, [S, H, D]
     uint16_t* qo; uint16_t* ko; uint16_t* vo;
     int64_t q_st, q_sh, k_st, k_sh, v_st, v_sh;
+    // to_streams != 0: the prepared rows go straight into the packed head-major streams of the attention kernels
+    // (text rows of q, k, v -> qt, kt, vt; summary rows of k, v, q -> ks_out, vs_out, qs_out) instead of qo / ko / vo:
+    // preparation and packing in one pass over q, k, v
+    int32_t to_streams;
+    uint16_t* qt; uint16_t* kt; uint16_t* vt; uint16_t* ks_out; uint16_t* vs_out; uint16_t* qs_out;
+    int64_t text_rows, summ_rows;
 };
 cudaError_t launch_prep(const PrepArgs& a, int64_t max_aug_len, int num_seqs, cudaStream_t stream);
+// Zeroes the padding rows of the packed streams (text: qt, kt, vt; summary: ks, vs, qs) that launch_prep in stream mode
+// does not write.
+cudaError_t launch_zero_stream_pads(const PrepArgs& a, int num_seqs, cudaStream_t stream);
+// Summary rows from the packed streams (query rows in qs): each attends to the keys of its own chunk.
+cudaError_t launch_summary_streams(const KernelArgs& a, const uint16_t* qs, cudaStream_t stream);
 
 }  // namespace ksa

@@ -38,13 +38,20 @@ __global__ void __launch_bounds__(256, kPrepMinBlocks) ksa_prep_kernel(PrepArgs 
     const int64_t full = (int64_t)sq.n_chunks * s_len;            // rows of the full chunks
     int pos;
     int64_t summ_index = -1;                                      // row of the summary projections, if a summary token
+    int64_t stream_row;                                           // row of the packed text or summary stream (stream mode)
     if (row_in_seq < full) {
         const int j = (int)(row_in_seq / s_len), off = (int)(row_in_seq - (int64_t)j * s_len);
-        if (off < a.k) pos = j * a.k + off;
-        else { pos = (j + 1) * a.k - 1; summ_index = (int64_t)sq.summ_base + (int64_t)j * a.m + (off - a.k); }
+        if (off < a.k) { pos = j * a.k + off; stream_row = (int64_t)sq.text_off + pos; }
+        else {
+            pos = (j + 1) * a.k - 1;
+            summ_index = (int64_t)sq.summ_base + (int64_t)j * a.m + (off - a.k);
+            stream_row = (int64_t)sq.summ_off + (int64_t)j * a.m + (off - a.k);
+        }
     } else {
         pos = sq.n_chunks * a.k + (int)(row_in_seq - full);       // text tokens after the last full chunk
+        stream_row = (int64_t)sq.text_off + pos;
     }
+    const bool is_summ = summ_index >= 0;
     const int64_t row = sq.aug_off + row_in_seq;
     // ---- the eight angles of this slice ---------------------------------------------------------
     const int d0 = slice * 8;
@@ -79,6 +86,10 @@ __global__ void __launch_bounds__(256, kPrepMinBlocks) ksa_prep_kernel(PrepArgs 
             if (which == 0)      { mainp = a.qm + row * a.q_st + (int64_t)h * a.q_sh; outp[u] = a.qo + row * a.q_st + (int64_t)h * a.q_sh; summp = a.qs; H = a.Hq; }
             else if (which == 1) { mainp = a.km + row * a.k_st + (int64_t)h * a.k_sh; outp[u] = a.ko + row * a.k_st + (int64_t)h * a.k_sh; summp = a.ks; H = a.Hkv; }
             else                 { mainp = a.vm + row * a.v_st + (int64_t)h * a.v_sh; outp[u] = a.vo + row * a.v_st + (int64_t)h * a.v_sh; summp = a.vs; H = a.Hkv; }
+            if (a.to_streams) {                                   // head-major streams: [head][row][D]
+                if (!is_summ) outp[u] = (which == 0 ? a.qt : (which == 1 ? a.kt : a.vt)) + ((int64_t)h * a.text_rows + stream_row) * a.D;
+                else          outp[u] = (which == 0 ? a.qs_out : (which == 1 ? a.ks_out : a.vs_out)) + ((int64_t)h * a.summ_rows + stream_row) * a.D;
+            }
             rotate[u] = a.rope && which != 2;
             lo[u] = *reinterpret_cast<const uint4*>(mainp + d0);
             hi[u] = *reinterpret_cast<const uint4*>(mainp + a.D / 2 + d0);
@@ -122,6 +133,36 @@ __global__ void __launch_bounds__(256, kPrepMinBlocks) ksa_prep_kernel(PrepArgs 
             *reinterpret_cast<uint4*>(outp[u] + a.D / 2 + d0) = ohi;
         }
     }
+}
+
+// Padding rows of the streams: rows [n_text, text_pad) of every sequence's part of qt, kt, vt and rows
+// [n_summ, summ_pad) of ks, vs, qs.  One block per (sequence, stream); at most 127 rows each.
+__global__ void __launch_bounds__(256) ksa_zero_stream_pads_kernel(PrepArgs a)
+{
+    const SeqInfo sq = a.seqs[blockIdx.y];
+    const int which = blockIdx.x;                                  // 0 qt, 1 kt, 2 vt, 3 ks_out, 4 vs_out, 5 qs_out
+    const bool text = which < 3;
+    uint16_t* base = which == 0 ? a.qt : which == 1 ? a.kt : which == 2 ? a.vt : which == 3 ? a.ks_out : which == 4 ? a.vs_out : a.qs_out;
+    const int H = (which == 0 || which == 5) ? a.Hq : a.Hkv;
+    const int64_t rows = text ? a.text_rows : a.summ_rows;
+    const int64_t r0 = text ? (int64_t)sq.text_off + sq.n_text : (int64_t)sq.summ_off + sq.n_summ;
+    const int64_t r1 = text ? (int64_t)sq.text_off + sq.text_pad : (int64_t)sq.summ_off + sq.summ_pad;
+    const int vecs = a.D / 8;
+    const int64_t total = (r1 - r0) * H * vecs;
+    for (int64_t idx = threadIdx.x; idx < total; idx += blockDim.x) {
+        const int vec = (int)(idx % vecs);
+        const int64_t t = idx / vecs;
+        const int h = (int)(t % H);
+        const int64_t row = r0 + t / H;
+        *reinterpret_cast<uint4*>(base + ((int64_t)h * rows + row) * a.D + vec * 8) = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+cudaError_t launch_zero_stream_pads(const PrepArgs& a, int num_seqs, cudaStream_t stream)
+{
+    dim3 grid(6u, (unsigned)num_seqs, 1u);
+    ksa_zero_stream_pads_kernel<<<grid, 256, 0, stream>>>(a);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_prep(const PrepArgs& a, int64_t max_aug_len, int num_seqs, cudaStream_t stream)

@@ -93,3 +93,64 @@ def test_prepare_in_place_and_whole_oracle(ctx):
 def test_anneal_lambda_matches_oracle():
     for step in (0, 99, 100, 101, 150, 299, 300, 10 ** 9):
         assert ksa.anneal_lambda(step, 100, 300) == pytest.approx(prep.anneal_lambda(step, 100, 300), abs=1e-7)
+
+
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D,lam,theta,flags", [
+    ([300, 77], 8, 1, 4, 4, 2, 128, 0.3, 1.0e4, 0),                  # ragged lengths
+    ([1024, 512], 8, 1, 16, 8, 2, 128, 0.6, 1.0e6, 0),               # whole chunks (the plain forward call would read these in place)
+    ([1500], 8, 1, 16, 8, 2, 128, 1.0, 1.0e6, 0),                    # several summary tiles
+    ([400, 130], 64, 8, 2, 4, 2, 128, 0.75, 1.0e4, 0),               # eight summaries per chunk
+    ([333], 3, 2, 5, 6, 2, 64, 0.5, 1.0e4, 0),                       # head_dim 64, odd group size
+    ([257], 16, 0, 3, 2, 2, 128, 0.5, 1.0e4, 0),                     # no summary tokens
+    ([200], 8, 1, 2, 4, 2, 128, 0.4, 0.0, ksa.KSA_PREP_NO_ROPE),     # interpolation only
+])
+def test_prepared_forward_equals_prepare_then_forward_and_the_oracles(ctx, lens, k, m, C, Hq, Hkv, D, lam, theta, flags):
+    """ksa_attn_fwd_prepared (preparation folded into the pack pass) against (a) ksa_qkv_prepare followed by ksa_attn_fwd:
+    the same arithmetic on the same rows, so the same bits, and (b) the two oracles chained: the fp64 preparation oracle,
+    rounded once to bf16 as the operator's inputs are, then the fp64 attention oracle."""
+    from oracle import ksa_oracle as orc
+    from tests import parity
+    dev = torch.device("cuda", 0)
+    scale = 1.0 / np.sqrt(D)
+    prob = ksa.Problem(lens, k, m, C, Hq, Hkv, D, scale, 0)
+    L, S = ksa.total_aug_len(prob), ksa.total_summary_rows(prob)
+    qm, km, vm = _rand((L, Hq, D), 11), _rand((L, Hkv, D), 12), _rand((L, Hkv, D), 13)
+    need_summ = lam != 0.0 and S > 0
+    qs, ks, vs = (_rand((S, Hq, D), 14), _rand((S, Hkv, D), 15), _rand((S, Hkv, D), 16)) if need_summ else (None, None, None)
+    to = lambda t: None if t is None else t.to(dev)
+    qd, kd, vd = qm.to(dev), km.to(dev), vm.to(dev)
+    # (a) two calls
+    qo, ko, vo = torch.empty_like(qd), torch.empty_like(kd), torch.empty_like(vd)
+    ctx.qkv_prepare(prob, qd, kd, vd, to(qs), to(ks), to(vs), qo, ko, vo, lam, theta, flags)
+    out2 = torch.empty_like(qd); lse2 = torch.empty((Hq, L), dtype=torch.float32, device=dev)
+    ws2 = torch.empty(max(256, ksa.workspace_bytes(prob)), dtype=torch.uint8, device=dev)
+    ctx.clear_device_status()
+    ctx.attn_fwd(prob, qo, ko, vo, out2, lse2, ws2)
+    # one call; canary-padded outputs, NaN-filled workspace
+    out = torch.full((L + 2, Hq, D), 7.0, dtype=torch.bfloat16, device=dev)
+    lse = torch.full((Hq * L + 64,), -5.0, dtype=torch.float32, device=dev)
+    out_v, lse_v = out[1:L + 1], lse[32:32 + Hq * L].view(Hq, L)
+    ws = torch.full((ksa.prepared_workspace_bytes(prob),), 0xFF, dtype=torch.uint8, device=dev)
+    ctx.attn_fwd_prepared(prob, qd, kd, vd, to(qs), to(ks), to(vs), lam, theta, out_v, lse_v, ws, flags)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert (out[0] == 7.0).all() and (out[-1] == 7.0).all() and (lse[:32] == -5.0).all() and (lse[-32:] == -5.0).all()
+    # text rows: the same tensor-core kernel on the same tiles -> the same bits; summary rows come from another kernel
+    is_summ = torch.from_numpy(prep.summary_rows(lens, k, m).astype(bool)).to(dev)
+    assert torch.equal(out_v[~is_summ], out2[~is_summ]) and torch.equal(lse_v[:, ~is_summ], lse2[:, ~is_summ])
+    # (b) the oracles
+    f64 = lambda t: None if t is None else t.double().numpy()
+    if flags & ksa.KSA_PREP_NO_ROPE:
+        pos, summ = prep.position_ids(lens, k, m), prep.summary_rows(lens, k, m)
+        idx = np.cumsum(summ) - 1
+        def blend(main, s_):
+            x = f64(main).copy()
+            if need_summ:
+                x[summ.astype(bool)] = lam * f64(s_)[idx[summ.astype(bool)]] + (1.0 - lam) * x[summ.astype(bool)]
+            return x
+        rq, rk, rv = blend(qm, qs), blend(km, ks), blend(vm, vs)
+    else:
+        rq, rk, rv = prep.prepare(f64(qm), f64(km), f64(vm), f64(qs), f64(ks), f64(vs), lens, k, m, lam if need_summ else 0.0, theta)
+    bits = lambda x: (torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+    ref_out, ref_lse, _ = orc.fwd(bits(rq), bits(rk), bits(rv), lens, k, m, C, scale)
+    parity.compare(out_v.double().cpu().numpy(), lse_v.double().cpu().numpy().T, ref_out, ref_lse, "prepared")
