@@ -534,55 +534,104 @@ __global__ void __launch_bounds__(256) ksa_text_ref_kernel(KernelArgs a)
 
 // ---------------------------------------------------------------------------------------
 // Summary rows from the packed streams (the path whose preparation pass wrote the streams directly, so that no
-// prepared interleaved tensors exist): one warp per (summary row, query head); lane l holds D / 32 elements.
-// Keys of summary (j, r): text rows [j k, j k + k) of the text stream, then summary rows j m .. j m + r of the
-// summary stream (Sec. 2.2.1; the latter not under KSA_FLAG_SUMMARY_TEXT_ONLY).  One key at a time, online softmax.
+// prepared interleaved tensors exist).  A warp takes one (summary row, KV head, round of four query heads): its four
+// groups of eight lanes each take one query head of the group, every lane D / 8 elements, so a dot product needs three
+// shuffle steps and the four groups read the same K / V addresses.  Keys of summary (j, r): text rows [j k, j k + k)
+// of the text stream, then summary rows j m .. j m + r of the summary stream (Sec. 2.2.1; the latter not under
+// KSA_FLAG_SUMMARY_TEXT_ONLY).  Keys go in batches of sixteen (all loads of a batch in flight together), with a
+// running maximum and sum across batches.
 // ---------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) ksa_summary_streams_kernel(KernelArgs a, const uint16_t* __restrict__ qs)
 {
-    constexpr int E = D / 32;
+    constexpr int E = D / 8;              // elements per lane
+    constexpr int V4 = E / 8;             // 16-byte vectors per lane
     const SeqInfo sq = a.seqs[blockIdx.y];
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, lg = lane >> 3, sub = lane & 7;
     const int G = a.Hq / a.Hkv;
-    const int64_t tasks = (int64_t)sq.n_summ * a.Hq;
+    const int rounds = (G + 3) / 4;
+    const int64_t tasks = (int64_t)sq.n_summ * a.Hkv * rounds;
     for (int64_t task = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); task < tasks; task += (int64_t)gridDim.x * 8) {
-        const int u = (int)(task / a.Hq), h = (int)(task % a.Hq), hk = h / G;
+        const int rd = (int)(task % rounds);
+        const int hk = (int)((task / rounds) % a.Hkv);
+        const int u = (int)(task / ((int64_t)rounds * a.Hkv));
         const int j = u / a.m, r = u % a.m;
+        const int gi = rd * 4 + lg;
+        const bool live = gi < G;
+        const int h = hk * G + (live ? gi : 0);
         float qv[E];
-        const uint16_t* qp = qs + ((int64_t)h * a.summ_rows + sq.summ_off + u) * D + lane * E;
+        {
+            const uint16_t* qp = qs + ((int64_t)h * a.summ_rows + sq.summ_off + u) * D + sub * E;
 #pragma unroll
-        for (int e = 0; e < E; ++e) qv[e] = __uint_as_float((uint32_t)qp[e] << 16);
+            for (int c = 0; c < V4; ++c) summ_unpack(*reinterpret_cast<const uint4*>(qp + 8 * c), qv + 8 * c);
+        }
         float mx = -INFINITY, l = 0.f, acc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
-        const int n_summ_keys = (a.flags & 0x1u) ? 0 : r + 1;
-        for (int t = 0; t < a.k + n_summ_keys; ++t) {
-            const bool text = t < a.k;
-            const int64_t row = text ? (int64_t)sq.text_off + (int64_t)j * a.k + t : (int64_t)sq.summ_off + (int64_t)j * a.m + (t - a.k);
-            const int64_t off = ((int64_t)hk * (text ? a.text_rows : a.summ_rows) + row) * D + lane * E;
-            const uint16_t* kp = (text ? a.kt : a.ks) + off;
-            const uint16_t* vp = (text ? a.vt : a.vs) + off;
-            float dot = 0.f;
+        const int nkeys = a.k + ((a.flags & 0x1u) ? 0 : r + 1);
+        const int64_t text0 = ((int64_t)hk * a.text_rows + sq.text_off + (int64_t)j * a.k) * D + sub * E;
+        const int64_t summ0 = ((int64_t)hk * a.summ_rows + sq.summ_off + (int64_t)j * a.m) * D + sub * E;
+        for (int c0 = 0; c0 < nkeys; c0 += 16) {
+            float sc[16];
 #pragma unroll
-            for (int e = 0; e < E; ++e) dot = fmaf(qv[e], __uint_as_float((uint32_t)kp[e] << 16), dot);
+            for (int t = 0; t < 16; ++t) {
+                const int key = c0 + t;
+                float dot = 0.f;
+                if (key < nkeys) {
+                    const uint16_t* kp = key < a.k ? a.kt + text0 + (int64_t)key * D : a.ks + summ0 + (int64_t)(key - a.k) * D;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            const float sc = dot * a.scale;
-            const float m_new = fmaxf(mx, sc);
-            const float corr = __expf(mx - m_new), p = __expf(sc - m_new);
-            l = l * corr + p;
+                    for (int c = 0; c < V4; ++c) {
+                        float kf[8];
+                        summ_unpack(*reinterpret_cast<const uint4*>(kp + 8 * c), kf);
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] = fmaf(p, __uint_as_float((uint32_t)vp[e] << 16), acc[e] * corr);
+                        for (int e = 0; e < 8; ++e) dot = fmaf(qv[8 * c + e], kf[e], dot);
+                    }
+                }
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                sc[t] = key < nkeys ? dot * a.scale : -INFINITY;
+            }
+            float cm = sc[0];
+#pragma unroll
+            for (int t = 1; t < 16; ++t) cm = fmaxf(cm, sc[t]);
+            const float m_new = fmaxf(mx, cm);
+            const float corr = __expf(mx - m_new);
+            l *= corr;
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] *= corr;
             mx = m_new;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const int key = c0 + t;
+                if (key < nkeys) {
+                    const float p = __expf(sc[t] - mx);
+                    l += p;
+                    const uint16_t* vp = key < a.k ? a.vt + text0 + (int64_t)key * D : a.vs + summ0 + (int64_t)(key - a.k) * D;
+#pragma unroll
+                    for (int c = 0; c < V4; ++c) {
+                        float vf[8];
+                        summ_unpack(*reinterpret_cast<const uint4*>(vp + 8 * c), vf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[8 * c + e] = fmaf(p, vf[e], acc[8 * c + e]);
+                    }
+                }
+            }
         }
         const int64_t aug = sq.aug_off + (int64_t)j * (a.k + a.m) + a.k + r;
-        if (ksa_out_row_ok(a, aug, h)) {
+        if (live && ksa_out_row_ok(a, aug, h)) {
             const float inv = 1.f / l;
-            uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + lane * E;
+            uint16_t* op = a.out + aug * a.o_st + (int64_t)h * a.o_sh + sub * E;
 #pragma unroll
-            for (int e = 0; e < E; ++e) op[e] = float_to_bf16_bits(acc[e] * inv);
-            if (lane == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
+            for (int c = 0; c < V4; ++c) {
+                uint4 ov;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&ov);
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    ow[e] = (uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e] * inv) | ((uint32_t)float_to_bf16_bits(acc[8 * c + 2 * e + 1] * inv) << 16);
+                *reinterpret_cast<uint4*>(op + 8 * c) = ov;
+            }
+            if (sub == 0) a.lse[(int64_t)h * a.total_aug + aug] = mx + __logf(l);
         }
     }
 }
@@ -590,7 +639,8 @@ __global__ void __launch_bounds__(256) ksa_summary_streams_kernel(KernelArgs a, 
 cudaError_t launch_summary_streams(const KernelArgs& a, const uint16_t* qs, cudaStream_t stream)
 {
     if (a.m <= 0 || a.max_n_summ <= 0) return cudaSuccess;
-    int64_t blocks = ((int64_t)a.max_n_summ * a.Hq + 7) / 8;
+    const int G = a.Hq / a.Hkv;
+    int64_t blocks = ((int64_t)a.max_n_summ * a.Hkv * ((G + 3) / 4) + 7) / 8;
     if (blocks > 148 * 32) blocks = 148 * 32;
     dim3 grid((unsigned)blocks, (unsigned)a.num_seqs, 1u);
     if (a.D == 128) ksa_summary_streams_kernel<128><<<grid, 256, 0, stream>>>(a, qs);
