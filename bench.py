@@ -264,7 +264,8 @@ def run_ours(args):
     wl, layout = workload_and_layout(args)
     if world > 1:   # independent batch per rank
         wl = dist_utils.rank_workload(wl, rank)
-    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale)
+    kflags = {"auto": 0, "single": ksa.KSA_FLAG_SINGLE_CTA_KERNEL, "pair": ksa.KSA_FLAG_CTA_PAIR_KERNEL}[args.text_kernel]
+    prob = ksa.Problem(wl.text_lens, layout.k, layout.m, layout.C, wl.Hq, wl.Hkv, wl.D, wl.scale, kflags)
     total = ksa.total_aug_len(prob)
     pairs = ksa.visible_pairs(prob)
     flops = 4.0 * wl.D * wl.Hq * pairs
@@ -372,14 +373,15 @@ def run_ours(args):
     text_flops = 4.0 * wl.D * wl.Hq * text_pairs
     text_avg_ms = sum(text_ms) / len(text_ms)
     achieved = text_flops / (text_avg_ms * 1e-3) / 1e12
-    traffic = ncu_traffic("ksa_text_tc_kernel", wl.name, layout.name)
+    kernel_name = "ksa_text_pair_kernel" if args.text_kernel == "pair" else "ksa_text_tc_kernel"
+    traffic = ncu_traffic(kernel_name, wl.name, layout.name)
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
         "frac": achieved / peaks["bf16_burst"], "traffic": traffic,
         "peak_source": f"of {peaks['source']} (burst bf16 GEMM rate: the dense BF16 tensor rate this box attains)",
         "frac_of_sustained_peak": achieved / peaks["bf16_sustained"], "sustained_peak": peaks["bf16_sustained"],
         "frac_of_nominal_2250": achieved / 2250.0,
-        "kernel": "ksa_text_tc_kernel", "kernel_ms_avg": text_avg_ms, "kernel_ms_median": statistics.median(text_ms),
+        "kernel": kernel_name, "kernel_ms_avg": text_avg_ms, "kernel_ms_median": statistics.median(text_ms),
         "kernel_ms_min": min(text_ms), "kernel_share_of_step": text_avg_ms / ms_per_step,
     }
 
@@ -727,6 +729,8 @@ def main():
     ap.add_argument("--workload", default="128k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--layout", default="P", choices=["P", "G", "F"],
                     help="P, G: the paper's KSA layouts; F: full causal attention (the hybrid stack's full layers)")
+    ap.add_argument("--text-kernel", default="auto", choices=["auto", "single", "pair"],
+                    help="text-row kernel: the library's choice, the one-CTA kernel, or the CTA-pair kernel (cta_group::2)")
     ap.add_argument("--oracle-rows", type=int, default=3000)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
