@@ -442,6 +442,8 @@ cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream)
         dim3 g2((unsigned)chunk_groups, ny, (unsigned)a.Hkv);
         if (a.D == 128) ksa_summary_short_kernel<128><<<g2, 256, 0, stream>>>(a);
         else            ksa_summary_short_kernel<64><<<g2, 256, 0, stream>>>(a);
+    } else if (summary_mma_applies(a)) {
+        return launch_summary_mma(a, max_chunks, ny, stream);
     } else {
         const int tasks = a.m * (a.Hq / a.Hkv);
         const int task_blocks = (tasks + kSummTaskBlock - 1) / kSummTaskBlock;

@@ -13,6 +13,10 @@ cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream);
 
 // Summary rows: each attends to the (at most k + m) keys of its own chunk.
 cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream);
+// The same for long chunks on mma.sync tiles: one block per (chunk, KV head); launch_summary dispatches to it when
+// summary_mma_applies (m G >= 8 query rows per block, at most 128 of them, at most 128 keys per chunk).
+bool summary_mma_applies(const KernelArgs& a);
+cudaError_t launch_summary_mma(const KernelArgs& a, int max_chunks, unsigned ny, cudaStream_t stream);
 
 // Text rows, CUDA-core cross-check kernel (KSA_FLAG_REFERENCE_KERNEL).
 cudaError_t launch_text_ref(const KernelArgs& a, cudaStream_t stream);
