@@ -73,6 +73,10 @@ extern "C" {
 /* Run the text rows through the CTA-pair kernel wherever it applies (see above), whatever the
  * library would pick by itself.  Ignored where it does not apply. */
 #define KSA_FLAG_CTA_PAIR_KERNEL     0x8u
+/* ksa_attn_bwd only: run dQ and dK / dV of the text rows through the mma.sync kernels (the first
+ * version of the backward pass) instead of the tcgen05 kernels.  Same results up to rounding
+ * order; several times slower; an on-device cross-check.  Ignored by the other calls. */
+#define KSA_FLAG_BWD_MMA_SYNC_KERNELS 0x10u
 
 typedef struct ksa_ctx ksa_ctx;    /* opaque */
 

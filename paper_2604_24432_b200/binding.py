@@ -26,6 +26,7 @@ KSA_FLAG_SUMMARY_TEXT_ONLY = 0x1
 KSA_FLAG_REFERENCE_KERNEL = 0x2
 KSA_FLAG_SINGLE_CTA_KERNEL = 0x4
 KSA_FLAG_CTA_PAIR_KERNEL = 0x8
+KSA_FLAG_BWD_MMA_SYNC_KERNELS = 0x10
 KSA_STREAM_TEXT, KSA_STREAM_SUMMARY = 0, 1
 
 EXPORTS = [

@@ -72,7 +72,8 @@ int validate(const ksa_params* p)
     if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
         return KSA_ERR_INVALID_ARG;
     if (p->reserved != 0) return KSA_ERR_INVALID_ARG;
-    if (p->flags & ~(KSA_FLAG_SUMMARY_TEXT_ONLY | KSA_FLAG_REFERENCE_KERNEL | KSA_FLAG_SINGLE_CTA_KERNEL | KSA_FLAG_CTA_PAIR_KERNEL)) return KSA_ERR_INVALID_ARG;
+    if (p->flags & ~(KSA_FLAG_SUMMARY_TEXT_ONLY | KSA_FLAG_REFERENCE_KERNEL | KSA_FLAG_SINGLE_CTA_KERNEL | KSA_FLAG_CTA_PAIR_KERNEL |
+                     KSA_FLAG_BWD_MMA_SYNC_KERNELS)) return KSA_ERR_INVALID_ARG;
     if (!(p->softmax_scale > 0.f) || !std::isfinite(p->softmax_scale)) return KSA_ERR_INVALID_ARG;
     if (p->cu_text_lens[0] != 0) return KSA_ERR_INVALID_ARG;
     for (int b = 0; b < p->num_seqs; ++b)
@@ -858,7 +859,7 @@ static BwdLayout bwd_layout(const ksa_params* p, const HostSchedule& hs)
 {
     BwdLayout b{};
     // no packed streams and no packed dO where the tensor-core kernels read the caller's tensors in place
-    const bool direct = p->head_dim == 128 && direct_ok(p);
+    const bool direct = p->head_dim == 128 && direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
     if (!direct) b.fwd = workspace_layout(p, hs);
     size_t off = b.fwd.total;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
@@ -910,7 +911,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     }
     // packed streams of the forward pass (text Q, K, V and summary K, V) -- not needed when the tensor-core kernels
     // can read whole tiles straight from the caller's tensors (the no-pack case of the forward pass)
-    const bool direct = p->head_dim == 128 && direct_ok(p);
+    const bool direct = p->head_dim == 128 && direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
     KernelArgs fa = make_args(ctx, p, q, k, v, dq /* unused */, const_cast<float*>(lse), workspace, bl.fwd);
     if (!direct && (e = launch_pack(fa, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     BwdArgs a{};
@@ -936,8 +937,8 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if (a.D == 128) {
-        // text rows on the tcgen05 tensor cores, fed by TMA from the packed streams
+    if (!(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS)) {
+        // text rows on the tcgen05 tensor cores, fed by TMA from the packed streams or the caller's tensors
         if (!ctx->bwd_tc_ready) {
             if ((e = setup_bwd_tc()) != cudaSuccess) return cuda_fail(ctx, e);
             ctx->bwd_tc_ready = true;

@@ -1,6 +1,6 @@
-// Backward pass of the text rows on the sm_100a tensor cores (head_dim 128): dK / dV and dQ.
+// Backward pass of the text rows on the sm_100a tensor cores (head_dim D = 128 or 64): dK / dV and dQ.
 //
-// Both kernels keep two 128 x 128 operand tiles resident in shared memory (A1, A2) and stream the tiles
+// Both kernels keep two 128 x D operand tiles resident in shared memory (A1, A2) and stream the tiles
 // of the other two operands (B1: three TMA-filled stages, B2: two) past them.  Per streamed tile j the
 // tensor pipe computes two products into TMEM, X_j = A1 B1_j^T and Y_j = A2 B2_j^T (128 x 128, fp32),
 // and the row warps turn them into bf16 operands for the accumulating MMAs in two phases:
@@ -50,19 +50,24 @@ using namespace ptx;
 constexpr int kBwdTcThreads = 576;
 constexpr int kBwdTcRegs = 96;                  // 18 warps: five on a scheduler, 5 x 32 x 96 registers fit its file
 constexpr int kBwdSegTiles = 16;                // dK / dV: query tiles (of 128 rows) per CTA
-constexpr int kBwdTileBytes = 128 * 128 * 2;    // one 128 x 128 bf16 tile: [d half][128 rows][128 B]
 constexpr int kB1Stages = 3, kB2Stages = 2;
 
-// shared memory map (bytes from the 1024-aligned base)
-constexpr int kOffA1 = 0, kOffA2 = kBwdTileBytes, kOffB1 = 2 * kBwdTileBytes, kOffB2 = kOffB1 + kB1Stages * kBwdTileBytes;
-constexpr int kOffBars = kOffB2 + kB2Stages * kBwdTileBytes;                          // 18 barriers
-constexpr int kOffMisc = kOffBars + 192;                                              // TMEM slot, abort flags
-constexpr int kOffRow = kOffMisc + 64;                                                // dK / dV: [2][lse, delta][128] per-query scalars
-constexpr int kBwdTcLayoutBytes = kOffRow + 2 * 2 * 128 * 4;
-constexpr int kBwdTcSmem = 232448;              // the whole opt-in window: the layout needs all but 768 bytes of it
+// shared memory map (bytes from the 1024-aligned base) for head_dim D
+template <int D>
+struct BtMap {
+    static constexpr int kTile = 128 * D * 2;   // one 128 x D bf16 tile: [64-element half of d][128 rows][128 B]
+    static constexpr int kOffA1 = 0, kOffA2 = kTile, kOffB1 = 2 * kTile, kOffB2 = kOffB1 + kB1Stages * kTile;
+    static constexpr int kOffBars = kOffB2 + kB2Stages * kTile;                        // 18 barriers
+    static constexpr int kOffMisc = kOffBars + 192;                                    // TMEM slot, abort flags
+    static constexpr int kOffRow = kOffMisc + 64;                                      // dK / dV: [2][lse, delta][128] per-query scalars
+    static constexpr int kLayoutBytes = kOffRow + 2 * 2 * 128 * 4;
+    // head_dim 128: the whole opt-in window (the layout needs all but 768 bytes of it); 64: the layout and the slack
+    // for its 1024-byte alignment
+    static constexpr int kSmem = D == 128 ? 232448 : kLayoutBytes + 1024;
+    static_assert(kLayoutBytes <= kSmem, "shared memory layout");
+};
 enum : int { BB_AFULL = 0, BB_B1FULL = 1, BB_B2FULL = 4, BB_XFULL = 6, BB_YFULL = 7, BB_PA = 8, BB_PB = 9, BB_OFULL = 10,
              BB_B1EMPTY = 11, BB_B2EMPTY = 14, BB_YFULL2 = 16, BB_PB2 = 17 };
-static_assert(kBwdTcLayoutBytes <= kBwdTcSmem, "shared memory layout");
 
 // Optional event trace (compile with -DKSA_BWD_TRACE=1 for the dQ kernel, =3 for the dK / dV kernel over summary
 // keys): one CTA records (event id, clock) pairs for lane 0 of every row warp; ksa_debug_read_bwd_trace() copies
@@ -123,31 +128,35 @@ __device__ __forceinline__ bool bt_wait_warp(uint32_t bar, uint32_t parity, uint
 }
 
 // Shared-memory layout and barrier addresses of one CTA.
+template <int D>
 struct BtSmem {
+    using M = BtMap<D>;
     uint32_t base;
-    __device__ __forceinline__ uint32_t a1() const { return base + kOffA1; }
-    __device__ __forceinline__ uint32_t a2() const { return base + kOffA2; }
-    __device__ __forceinline__ uint32_t b1(int stage) const { return base + kOffB1 + (uint32_t)stage * kBwdTileBytes; }
-    __device__ __forceinline__ uint32_t b2(int stage) const { return base + kOffB2 + (uint32_t)stage * kBwdTileBytes; }
-    __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBars + 8u * (uint32_t)i; }
-    __device__ __forceinline__ uint32_t tmem_slot() const { return base + kOffMisc; }
-    __device__ __forceinline__ uint32_t abort_addr() const { return base + kOffMisc + 4; }
+    __device__ __forceinline__ uint32_t a1() const { return base + M::kOffA1; }
+    __device__ __forceinline__ uint32_t a2() const { return base + M::kOffA2; }
+    __device__ __forceinline__ uint32_t b1(int stage) const { return base + M::kOffB1 + (uint32_t)stage * M::kTile; }
+    __device__ __forceinline__ uint32_t b2(int stage) const { return base + M::kOffB2 + (uint32_t)stage * M::kTile; }
+    __device__ __forceinline__ uint32_t bar(int i) const { return base + M::kOffBars + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t tmem_slot() const { return base + M::kOffMisc; }
+    __device__ __forceinline__ uint32_t abort_addr() const { return base + M::kOffMisc + 4; }
 };
 
 // The layout starts on the first 1024-byte boundary of the dynamic window; false (and a status code) if it
 // does not fit behind it.  Uniform over the CTA: everybody returns before any barrier is touched.
-__device__ __forceinline__ bool bt_layout(BtSmem& sm, const uint8_t* raw, int32_t* status)
+template <int D>
+__device__ __forceinline__ bool bt_layout(BtSmem<D>& sm, const uint8_t* raw, int32_t* status)
 {
     const uint32_t raw_addr = smem_u32(raw);
     sm.base = (raw_addr + 1023u) & ~1023u;
-    if (sm.base - raw_addr + (uint32_t)kBwdTcLayoutBytes > (uint32_t)kBwdTcSmem) {
+    if (sm.base - raw_addr + (uint32_t)BtMap<D>::kLayoutBytes > (uint32_t)BtMap<D>::kSmem) {
         if (threadIdx.x == 0) atomicCAS(status, 0, (int)kStatusSmemLayout);
         return false;
     }
     return true;
 }
 
-__device__ __forceinline__ void bt_init(const BtSmem& sm, int tid, int warp)
+template <int D>
+__device__ __forceinline__ void bt_init(const BtSmem<D>& sm, int tid, int warp)
 {
     if (tid == 0) {
         mbar_init(sm.bar(BB_AFULL), 1);
@@ -171,23 +180,25 @@ __device__ __forceinline__ void bt_init(const BtSmem& sm, int tid, int warp)
 }
 
 // ---- MMA issue helpers (one thread) ---------------------------------------------------------------
-// D[tmem_d] = A B^T, both 128 x 128 tiles K-major in shared memory ([d half][128 rows][128 B]).
+// D[tmem_d] = A B^T, both 128 x D tiles K-major in shared memory ([64-element half of d][128 rows][128 B]).
+template <int D>
 __device__ __forceinline__ void bt_product(uint32_t tmem_d, uint32_t a_tile, uint32_t b_tile)
 {
     constexpr uint32_t idesc = make_idesc_bf16(128, 128, false);
     const uint64_t ad = make_smem_desc_sw128(a_tile, 16, 1024), bd = make_smem_desc_sw128(b_tile, 16, 1024);
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
+    for (int kk = 0; kk < D / 16; ++kk) {
         const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
         mma_ss(tmem_d, ad + off, bd + off, idesc, kk > 0 ? 1u : 0u);
     }
 }
 // D[tmem_d] (+)= A B: A = 128 x 128 bf16 in TMEM (16 packed columns at the start of every 32-column chunk of
-// tmem_a), B = a 128 x 128 tile in shared memory read MN-major (64-element atoms of d 16384 bytes apart,
-// 8-row groups 1024 bytes apart).
+// tmem_a), B = a 128 x D tile in shared memory read MN-major (64-element atoms of d 16384 bytes apart,
+// 8-row groups 1024 bytes apart): D accumulator columns.
+template <int D>
 __device__ __forceinline__ void bt_accumulate(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_tile, bool first)
 {
-    constexpr uint32_t idesc = make_idesc_bf16(128, 128, true);
+    constexpr uint32_t idesc = make_idesc_bf16(128, D, true);
     const uint64_t bd = make_smem_desc_sw128(b_tile, 16384, 1024);
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk)
@@ -197,9 +208,10 @@ __device__ __forceinline__ void bt_accumulate(uint32_t tmem_d, uint32_t tmem_a, 
 // Half of such an accumulation for the dK / dV kernel, whose row warps hand their 32-column blocks over in two
 // halves of 16 query columns: the four k-steps 2 c + odd, whose 16 x bf16 operand stands in the 8 columns at
 // tmem_a + 32 c + 16 odd (tmem_a already points at dS^T, or 8 columns further at P^T).
+template <int D>
 __device__ __forceinline__ void bt_accumulate_half(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_tile, int odd, bool first)
 {
-    constexpr uint32_t idesc = make_idesc_bf16(128, 128, true);
+    constexpr uint32_t idesc = make_idesc_bf16(128, D, true);
     const uint64_t bd = make_smem_desc_sw128(b_tile, 16384, 1024);
 #pragma unroll
     for (int c = 0; c < 4; ++c)
@@ -210,24 +222,27 @@ __device__ __forceinline__ void bt_accumulate_half(uint32_t tmem_d, uint32_t tme
 // The two 64-column halves of a 128-row tile.  Packed streams: rows pos .. pos + 127 of a 3-D map.  Direct mode
 // (no packed copies: every sequence a whole number of chunks): chunks pos .. of a 4-D view [D, rows per chunk,
 // chunk, head] of the caller's interleaved tensor, whose box lands in shared memory as the same dense tile.
+template <int D>
 __device__ __forceinline__ void bt_issue_tile(uint32_t dst, uint32_t bar, const CUtensorMap* map, int pos, int head, bool direct)
 {
     if (direct) {
         tma_load_4d(dst, map, bar, 0, 0, pos, head);
-        tma_load_4d(dst + 16384, map, bar, 64, 0, pos, head);
+        if (D == 128) tma_load_4d(dst + 16384, map, bar, 64, 0, pos, head);
     } else {
         tma_load_3d(dst, map, bar, 0, pos, head);
-        tma_load_3d(dst + 16384, map, bar, 64, pos, head);
+        if (D == 128) tma_load_3d(dst + 16384, map, bar, 64, pos, head);
     }
 }
+template <int D>
 __device__ __forceinline__ void bt_load_tile(uint32_t dst, uint32_t bar, const CUtensorMap* map, int pos, int head, bool direct)
 {
-    mbar_arrive_expect_tx(bar, (uint32_t)kBwdTileBytes);
-    bt_issue_tile(dst, bar, map, pos, head, direct);
+    mbar_arrive_expect_tx(bar, (uint32_t)BtMap<D>::kTile);
+    bt_issue_tile<D>(dst, bar, map, pos, head, direct);
 }
 // After an abort: leave no copy in flight.  Bounded waits (the second flag is never set) for the last fill of
 // every stage; filled1 / filled2 = B1 / B2 tiles whose load was issued.
-__device__ __forceinline__ void bt_drain(const BtSmem& sm, int filled1, int filled2, int32_t* status)
+template <int D>
+__device__ __forceinline__ void bt_drain(const BtSmem<D>& sm, int filled1, int filled2, int32_t* status)
 {
     const uint32_t never = sm.abort_addr() + 4;
     bt_wait(sm.bar(BB_AFULL), 0, never, status, kStatusWaitKvFull);
@@ -242,7 +257,8 @@ __device__ __forceinline__ void bt_drain(const BtSmem& sm, int filled1, int fill
 }
 
 // Stage `stage` (of `stages`) is about to take tile j: wait until its previous tile (j - stages) was released.
-__device__ __forceinline__ bool bt_stage_free(const BtSmem& sm, int empty0, int stages, int j, int32_t* status)
+template <int D>
+__device__ __forceinline__ bool bt_stage_free(const BtSmem<D>& sm, int empty0, int stages, int j, int32_t* status)
 {
     if (j < stages) return true;
     return bt_wait(sm.bar(empty0 + j % stages), (uint32_t)((j / stages - 1) & 1), sm.abort_addr(), status, kStatusWaitQEmpty);
@@ -251,6 +267,7 @@ __device__ __forceinline__ bool bt_stage_free(const BtSmem& sm, int empty0, int 
 // =====================================================================================================
 // dK / dV
 // =====================================================================================================
+template <int D>
 __global__ void __maxnreg__(kBwdTcRegs)
 ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ)
 {
@@ -284,13 +301,13 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
     const int krow0 = (summ ? sq.summ_off : sq.text_off) + kt * 128;      // first row of the key tile in its packed stream
     auto pair_of = [&](int j, int& qt, int& h) { qt = seg0 + j / G; h = hk * G + j % G; };
 
-    BtSmem sm;
+    BtSmem<D> sm;
     if (!bt_layout(sm, bsm_raw, a.status)) return;
     uint8_t* base_ptr = bsm_raw + (sm.base - smem_u32(bsm_raw));
     // per-query scalars of the streamed tile, double-buffered by j: [j & 1][lse, delta][128 columns]; every row
     // warp writes the 32 columns it reads itself, one tile ahead (the four warps of a column group write the same
     // values, and each relies on its own writes only), see below
-    float* rows = reinterpret_cast<float*>(base_ptr + kOffRow);
+    float* rows = reinterpret_cast<float*>(base_ptr + BtMap<D>::kOffRow);
     const int quarter = warp & 3, cg = warp >> 2;                        // row warps: lanes 32 quarter ..; columns 32 cg ..
     const bool scalar_writer = warp < 16 && quarter == 0;
     float n_lse = 0.f, n_dl = 0.f;                                        // the writer lane's values for the next tile
@@ -315,11 +332,11 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             prefetch_tensormap(&maps.qt); prefetch_tensormap(&maps.dot);
             const bool direct = a.direct != 0;
             const int q_step = direct ? 128 / a.k : 128, q_base = direct ? sq.chunk0 : sq.text_off;   // position of a query tile
-            mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * kBwdTileBytes);
+            mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * BtMap<D>::kTile);
             {
                 const int kpos = direct ? sq.chunk0 + kt * (128 / (summ ? a.m : a.k)) : krow0;
-                bt_issue_tile(sm.a1(), sm.bar(BB_AFULL), summ ? &maps.ks : &maps.kt, kpos, hk, direct);
-                bt_issue_tile(sm.a2(), sm.bar(BB_AFULL), summ ? &maps.vs : &maps.vt, kpos, hk, direct);
+                bt_issue_tile<D>(sm.a1(), sm.bar(BB_AFULL), summ ? &maps.ks : &maps.kt, kpos, hk, direct);
+                bt_issue_tile<D>(sm.a2(), sm.bar(BB_AFULL), summ ? &maps.vs : &maps.vt, kpos, hk, direct);
             }
             int filled1 = 0, filled2 = 0;
             bool ok = true;
@@ -328,10 +345,10 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                 pair_of(j, qt, h);
                 const int pos = q_base + qt * q_step;
                 if (!(ok = bt_stage_free(sm, BB_B1EMPTY, kB1Stages, j, a.status))) break;
-                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), &maps.qt, pos, h, direct);
+                bt_load_tile<D>(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), &maps.qt, pos, h, direct);
                 ++filled1;
                 if (!(ok = bt_stage_free(sm, BB_B2EMPTY, kB2Stages, j, a.status))) break;
-                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), &maps.dot, pos, h, direct);
+                bt_load_tile<D>(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), &maps.dot, pos, h, direct);
                 ++filled2;
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, filled1, filled2, a.status);
@@ -342,9 +359,9 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
             const uint32_t abort_addr = sm.abort_addr();
             bool alive = bt_wait(sm.bar(BB_AFULL), 0, abort_addr, a.status, kStatusWaitKvFull);
             if (alive) alive = bt_wait(sm.bar(BB_B1FULL), 0, abort_addr, a.status, kStatusWaitQFull);
-            if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
+            if (alive) { bt_product<D>(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
-            if (alive) { bt_product(tY, sm.a2(), sm.b2(0)); tc_commit(sm.bar(BB_YFULL)); }
+            if (alive) { bt_product<D>(tY, sm.a2(), sm.b2(0)); tc_commit(sm.bar(BB_YFULL)); }
             uint32_t bt_wait_a = 0, bt_wait_b = 0, bt_wait_c = 0, bt_iss_x = 0, bt_iss_acc = 0;
             const uint32_t bt_loop0 = (uint32_t)clock();
             (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0; (void)bt_wait_c; (void)bt_iss_x; (void)bt_iss_acc;
@@ -360,7 +377,7 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                     if (!bt_wait(sm.bar(BB_B1FULL + s1), ((j + 1) / kB1Stages) & 1, abort_addr, a.status, kStatusWaitQFull)) break;
                     KSA_BT_WAIT_END(bt_wait_c); }
                     { KSA_BT_WAIT_BEGIN();
-                    bt_product(tX, sm.a1(), sm.b1(s1));
+                    bt_product<D>(tX, sm.a1(), sm.b1(s1));
                     tc_commit(sm.bar(BB_XFULL));
                     KSA_BT_WAIT_END(bt_iss_x); }
                 }
@@ -370,16 +387,16 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                   KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
                 KSA_BT_WAIT_BEGIN();
-                bt_accumulate_half(tDV, tY + 8, sm.b2(j & 1), 0, j == 0);                   // dV += P^T dO_j
-                bt_accumulate_half(tDK, tY, sm.b1(j % kB1Stages), 0, j == 0);               // dK += dS^T Q_j
+                bt_accumulate_half<D>(tDV, tY + 8, sm.b2(j & 1), 0, j == 0);                   // dV += P^T dO_j
+                bt_accumulate_half<D>(tDK, tY, sm.b1(j % kB1Stages), 0, j == 0);               // dK += dS^T Q_j
                 // ... the other 16 (row warp 0 checked the stage of Y_{j+1} before it arrived): the odd k-steps
                 if (!bt_wait(sm.bar(BB_PB2), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                 tc_fence_after();
-                bt_accumulate_half(tDV, tY + 8, sm.b2(j & 1), 1, false);
+                bt_accumulate_half<D>(tDV, tY + 8, sm.b2(j & 1), 1, false);
                 tc_commit(sm.bar(BB_B2EMPTY + (j & 1)));                                    // ... then its dO stage is free
-                bt_accumulate_half(tDK, tY, sm.b1(j % kB1Stages), 1, false);
+                bt_accumulate_half<D>(tDK, tY, sm.b1(j % kB1Stages), 1, false);
                 tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // ... then its Q stage is free
-                if (j + 1 < J) { bt_product(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
+                if (j + 1 < J) { bt_product<D>(tY, sm.a2(), sm.b2((j + 1) & 1)); tc_commit(sm.bar(BB_YFULL)); }
                 KSA_BT_WAIT_END(bt_iss_acc);
             }
             tc_commit(sm.bar(BB_OFULL));
@@ -518,16 +535,16 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
 #endif
         if (alive && bt_wait_warp(sm.bar(BB_OFULL), 0, sm.abort_addr(), a.status, kStatusWaitOFull, lane)) {
             tc_fence_after();
-            // odd cg: scale * dK, even cg: dV; cg / 2 picks the 64-element half of the row
+            // odd cg: scale * dK, even cg: dV; cg / 2 picks the half of the row (D / 2 elements)
             // (tcgen05.ld is warp-collective: rows past the stream load, too)
             const bool is_dk = (cg & 1) != 0;
-            const int d0 = (cg >> 1) * 64;
+            const int d0 = (cg >> 1) * (D / 2);
             const size_t arow = (size_t)hk * (summ ? a.summ_rows : a.text_rows) + (size_t)krow0 + quarter * 32 + lane;
-            float* acc = (is_dk ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * 128 + d0;
+            float* acc = (is_dk ? (summ ? a.dks : a.dkt) : (summ ? a.dvs : a.dvt)) + arow * D + d0;
             const float mul = is_dk ? a.scale : 1.f;
             const uint32_t tacc = (is_dk ? tDK : tDV) + lane_sel + d0;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < D / 64; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tacc + c * 32, o);
                 tc_wait_ld();
@@ -549,6 +566,7 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
 // =====================================================================================================
 // dQ
 // =====================================================================================================
+template <int D>
 __global__ void __maxnreg__(kBwdTcRegs)
 ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps)
 {
@@ -572,7 +590,7 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         key0 = (is_summ ? j : t_lo + j - n_s) * 128;
     };
 
-    BtSmem sm;
+    BtSmem<D> sm;
     if (!bt_layout(sm, bsm_raw, a.status)) return;
     bt_init(sm, tid, warp);
     const uint32_t tmem = bt_ld_shared(sm.tmem_slot());
@@ -588,11 +606,11 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
         if (lane == 0) {
             prefetch_tensormap(&maps.kt); prefetch_tensormap(&maps.vt);
             const bool direct = a.direct != 0;
-            mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * kBwdTileBytes);
+            mbar_arrive_expect_tx(sm.bar(BB_AFULL), 2u * BtMap<D>::kTile);
             {
                 const int qpos = direct ? sq.chunk0 + qt * (128 / a.k) : sq.text_off + qt * 128;
-                bt_issue_tile(sm.a1(), sm.bar(BB_AFULL), &maps.qt, qpos, h, direct);
-                bt_issue_tile(sm.a2(), sm.bar(BB_AFULL), &maps.dot, qpos, h, direct);
+                bt_issue_tile<D>(sm.a1(), sm.bar(BB_AFULL), &maps.qt, qpos, h, direct);
+                bt_issue_tile<D>(sm.a2(), sm.bar(BB_AFULL), &maps.dot, qpos, h, direct);
             }
             int filled1 = 0, filled2 = 0;
             bool ok = true;
@@ -603,10 +621,10 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
                 const int pos = direct ? sq.chunk0 + (key0 >> 7) * (128 / (is_summ ? a.m : a.k))
                                        : (is_summ ? sq.summ_off : sq.text_off) + key0;
                 if (!(ok = bt_stage_free(sm, BB_B1EMPTY, kB1Stages, j, a.status))) break;
-                bt_load_tile(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), is_summ ? &maps.ks : &maps.kt, pos, hk, direct);
+                bt_load_tile<D>(sm.b1(j % kB1Stages), sm.bar(BB_B1FULL + j % kB1Stages), is_summ ? &maps.ks : &maps.kt, pos, hk, direct);
                 ++filled1;
                 if (!(ok = bt_stage_free(sm, BB_B2EMPTY, kB2Stages, j, a.status))) break;
-                bt_load_tile(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), is_summ ? &maps.vs : &maps.vt, pos, hk, direct);
+                bt_load_tile<D>(sm.b2(j & 1), sm.bar(BB_B2FULL + (j & 1)), is_summ ? &maps.vs : &maps.vt, pos, hk, direct);
                 ++filled2;
             }
             if (bt_ld_shared(sm.abort_addr()) != 0u) bt_drain(sm, filled1, filled2, a.status);
@@ -617,9 +635,9 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             const uint32_t abort_addr = sm.abort_addr();
             bool alive = bt_wait(sm.bar(BB_AFULL), 0, abort_addr, a.status, kStatusWaitKvFull);
             if (alive) alive = bt_wait(sm.bar(BB_B1FULL), 0, abort_addr, a.status, kStatusWaitQFull);
-            if (alive) { bt_product(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
+            if (alive) { bt_product<D>(tX, sm.a1(), sm.b1(0)); tc_commit(sm.bar(BB_XFULL)); }
             if (alive) alive = bt_wait(sm.bar(BB_B2FULL), 0, abort_addr, a.status, kStatusWaitQFull);
-            if (alive) { bt_product(tY(0), sm.a2(), sm.b2(0)); tc_commit(y_full(0)); }
+            if (alive) { bt_product<D>(tY(0), sm.a2(), sm.b2(0)); tc_commit(y_full(0)); }
             uint32_t bt_wait_a = 0, bt_wait_b = 0;
             const uint32_t bt_loop0 = (uint32_t)clock();
             (void)bt_wait_a; (void)bt_wait_b; (void)bt_loop0;
@@ -631,16 +649,16 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
                     if (!bt_wait(sm.bar(BB_PA), j & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                     KSA_BT_WAIT_END(bt_wait_a);
                     tc_fence_after();
-                    bt_product(tX, sm.a1(), sm.b1((j + 1) % kB1Stages));
+                    bt_product<D>(tX, sm.a1(), sm.b1((j + 1) % kB1Stages));
                     tc_commit(sm.bar(BB_XFULL));
-                    bt_product(tY(j + 1), sm.a2(), sm.b2((j + 1) & 1));
+                    bt_product<D>(tY(j + 1), sm.a2(), sm.b2((j + 1) & 1));
                     tc_commit(y_full(j + 1));
                 }
                 { KSA_BT_WAIT_BEGIN();
                   if (!bt_wait(p_b(j), (j >> 1) & 1, abort_addr, a.status, kStatusWaitPFull)) break;
                   KSA_BT_WAIT_END(bt_wait_b); }
                 tc_fence_after();
-                bt_accumulate(tDQ, tY(j), sm.b1(j % kB1Stages), j == 0);                    // dQ += dS K_j
+                bt_accumulate<D>(tDQ, tY(j), sm.b1(j % kB1Stages), j == 0);                    // dQ += dS K_j
                 tc_commit(sm.bar(BB_B1EMPTY + j % kB1Stages));                              // K_j is free after that
             }
             tc_commit(sm.bar(BB_OFULL));
@@ -776,9 +794,11 @@ ksa_bwd_dq_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ 
             const int64_t aug = sq.aug_off + (int64_t)iq * (a.k + a.m) + (i - iq * a.k);
             uint16_t* dst = a.dq + aug * a.dq_st + (int64_t)h * a.dq_sh + cg * 32;
             uint32_t o[32];
-            tmem_ld32(tDQ + lane_sel + cg * 32, o);
-            tc_wait_ld();
-            if (i < sq.n_text) {
+            if (cg * 32 < D) {                                            // warp-uniform: the row has D elements
+                tmem_ld32(tDQ + lane_sel + cg * 32, o);
+                tc_wait_ld();
+            }
+            if (cg * 32 < D && i < sq.n_text) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
                     uint4 w;
@@ -808,15 +828,18 @@ extern "C" __attribute__((visibility("default"))) int ksa_debug_read_bwd_trace(v
 
 cudaError_t setup_bwd_tc()
 {
-    cudaError_t e = cudaFuncSetAttribute(ksa_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdTcSmem);
+    cudaError_t e = cudaFuncSetAttribute(ksa_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BtMap<128>::kSmem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(ksa_bwd_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdTcSmem);
+    if ((e = cudaFuncSetAttribute(ksa_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BtMap<128>::kSmem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(ksa_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BtMap<64>::kSmem)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(ksa_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BtMap<64>::kSmem);
 }
 
 cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream)
 {
     dim3 grid((unsigned)(a.max_text_pad / 128), (unsigned)a.Hq, (unsigned)a.num_seqs);
-    ksa_bwd_dq_tc_kernel<<<grid, kBwdTcThreads, kBwdTcSmem, stream>>>(a, maps);
+    if (a.D == 128) ksa_bwd_dq_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps);
+    else            ksa_bwd_dq_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps);
     return cudaGetLastError();
 }
 
@@ -829,7 +852,8 @@ cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_
         const long long span = summ ? n_qt : text_span;
         const int tiles = summ ? (a.max_n_summ + 127) / 128 : n_qt;
         dim3 grid((unsigned)((span + kBwdSegTiles - 1) / kBwdSegTiles), (unsigned)tiles, (unsigned)(a.num_seqs * a.Hkv));
-        ksa_bwd_dkv_tc_kernel<<<grid, kBwdTcThreads, kBwdTcSmem, stream>>>(a, maps, summ);
+        if (a.D == 128) ksa_bwd_dkv_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps, summ);
+        else            ksa_bwd_dkv_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps, summ);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

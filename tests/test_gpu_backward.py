@@ -51,6 +51,16 @@ def _check(name, got, ref):
     ([640], 8, 1, 3, 4, 1, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
     ([500], 8, 3, 2, 4, 2, 128, 0),                   # three summaries per chunk: packed streams, 128 % m != 0
     ([400, 136], 8, 1, 2, 4, 4, 128, 0),              # one query head per KV head, with summaries
+    # head_dim 64 on the tcgen05 kernels
+    ([1000, 300], 8, 1, 16, 8, 2, 64, 0),
+    ([2500], 64, 8, 4, 4, 2, 64, 0),
+    ([2100, 640], 8, 1, 16, 4, 4, 64, 0),
+    ([700], 16, 0, 7, 4, 4, 64, 0),
+    ([450], 8, 1, 3, 4, 1, 64, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
+    # the mma.sync kernels (the on-device cross-check of the tcgen05 kernels)
+    ([1000], 8, 1, 16, 8, 2, 128, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
+    ([520, 130], 3, 2, 5, 6, 2, 64, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
+    ([1024, 264, 8], 8, 1, 4, 4, 2, 128, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
 ])
 def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
     wl = synth.Workload("bwd", 31, lens, Hq, Hkv, D)
@@ -71,7 +81,7 @@ def test_backward_matches_oracle(ctx, lens, k, m, C, Hq, Hkv, D, flags):
         ctx.attn_bwd(prob, qd, kd, vd, out, lse, gd, dq, dk, dv, wsb)
     torch.cuda.synchronize()
     assert ctx.device_status() == 0
-    oflags = orc.SUMMARY_TEXT_ONLY if flags else 0
+    oflags = orc.SUMMARY_TEXT_ONLY if (flags & ksa.KSA_FLAG_SUMMARY_TEXT_ONLY) else 0
     rdq, rdk, rdv = orc.bwd(synth.bits(q), synth.bits(kk), synth.bits(v), synth.bits(dout), lens, k, m, C, wl.scale, oflags)
     _check("dq", dq.double().cpu().numpy(), rdq)
     _check("dk", dk.double().cpu().numpy(), rdk)
