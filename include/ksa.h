@@ -184,7 +184,7 @@ int ksa_attn_fwd_part(ksa_ctx* ctx, const void* q, const void* k, const void* v,
 /* ---- backward ----------------------------------------------------------------------- */
 /* Bytes of DEVICE workspace ksa_attn_bwd needs for this problem: the fp32 accumulators of dK / dV and two fp32
  * scalars per text row and query head, plus packed copies of q, k, v and dout unless they can be read in place
- * (head_dim 128 and every sequence a whole number of chunks). */
+ * (every sequence a whole number of chunks, 128 a multiple of the chunk length and of the summaries per chunk). */
 int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* bytes);
 /*
  * Gradients of ksa_attn_fwd (the kernel of Sec. 2.3 is the one "for training and prefill"):
@@ -198,8 +198,8 @@ int ksa_bwd_workspace_bytes(const ksa_ctx* ctx, const ksa_params* p, size_t* byt
  *   dk, dv              DEVICE bf16, layouts and strides of k and v; every row is written
  *   workspace           DEVICE, >= ksa_bwd_workspace_bytes, 256-byte aligned, scratch
  * Asynchronous on cuda_stream.  KSA_FLAG_REFERENCE_KERNEL is not accepted here.
- * With head_dim 128 and every sequence a whole number of chunks (the no-pack case of
- * ksa_attn_fwd) the tensor-core kernels read q, k, v and dout in place: rows of other
+ * With every sequence a whole number of chunks (the no-pack case of ksa_attn_fwd) the
+ * tensor-core kernels read q, k, v and dout in place: rows of other
  * sequences that share a 128-row tile are masked, so all of these tensors must hold finite
  * values everywhere.
  * Errors as for ksa_attn_fwd.

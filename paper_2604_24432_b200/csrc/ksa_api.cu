@@ -859,7 +859,7 @@ static BwdLayout bwd_layout(const ksa_params* p, const HostSchedule& hs)
 {
     BwdLayout b{};
     // no packed streams and no packed dO where the tensor-core kernels read the caller's tensors in place
-    const bool direct = p->head_dim == 128 && direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
+    const bool direct = direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
     if (!direct) b.fwd = workspace_layout(p, hs);
     size_t off = b.fwd.total;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
@@ -911,7 +911,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     }
     // packed streams of the forward pass (text Q, K, V and summary K, V) -- not needed when the tensor-core kernels
     // can read whole tiles straight from the caller's tensors (the no-pack case of the forward pass)
-    const bool direct = p->head_dim == 128 && direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
+    const bool direct = direct_ok(p) && !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS);
     KernelArgs fa = make_args(ctx, p, q, k, v, dq /* unused */, const_cast<float*>(lse), workspace, bl.fwd);
     if (!direct && (e = launch_pack(fa, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     BwdArgs a{};

@@ -57,6 +57,8 @@ def _check(name, got, ref):
     ([2100, 640], 8, 1, 16, 4, 4, 64, 0),
     ([700], 16, 0, 7, 4, 4, 64, 0),
     ([450], 8, 1, 3, 4, 1, 64, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
+    ([1024, 264, 8], 8, 1, 4, 4, 2, 64, 0),           # whole chunks: read in place
+    ([1280], 64, 8, 4, 4, 2, 64, 0),
     # the mma.sync kernels (the on-device cross-check of the tcgen05 kernels)
     ([1000], 8, 1, 16, 8, 2, 128, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
     ([520, 130], 3, 2, 5, 6, 2, 64, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
