@@ -95,6 +95,22 @@ def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), kernel_flag)
 
 
+@pytest.mark.parametrize("strict", [0, STRICT])
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
+    ([700, 200], 24, 3, 2, 12, 2, 128),    # 18 query rows per chunk and KV head (two 16-row tiles, one ragged), 27 keys
+    ([1000], 120, 8, 1, 16, 1, 128),       # the largest block: 128 query rows (eight tiles for four warps), 128 keys
+    ([600], 56, 8, 1, 4, 4, 64),           # one query head per KV head, head_dim 64
+    ([512, 40], 13, 8, 3, 8, 2, 128),      # odd chunk length, a sequence of three chunks and a tail
+    ([300], 16, 2, 2, 8, 2, 128),          # the smallest block: 8 query rows, 18 keys
+])
+def test_summary_rows_on_mma_tiles(ctx, lens, k, m, C, Hq, Hkv, D, strict):
+    """Chunks longer than the short-chunk kernel takes, with at least 8 (summary row, query head) pairs per chunk and KV
+    head and at most 128 of them and 128 keys: the summary rows run on the mma.sync kernel.  Every row against the oracle,
+    with and without the chunk's own summaries visible (Sec. 2.2.1)."""
+    wl = synth.Workload("summ-mma", 97, lens, Hq, Hkv, D)
+    parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), strict)
+
+
 @pytest.mark.parametrize("lens,k,m,C,Hq,Hkv", [
     ([1], 8, 1, 2, 2, 1), ([7], 8, 1, 2, 2, 1), ([127, 129, 128], 8, 1, 3, 4, 2), ([333, 1000], 3, 2, 5, 4, 2),
     ([777], 16, 0, 7, 4, 2), ([640], 1, 1, 100, 2, 1), ([1290], 200, 3, 1, 4, 1), ([2048, 640, 1336], 8, 1, 16, 8, 2),
