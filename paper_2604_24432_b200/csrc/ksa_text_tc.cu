@@ -255,7 +255,10 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                         if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
                     }
                     KSA_TR(0, 39);
+                    // both stages of this iteration are checked here, while the softmax warps still work on P_0: the ring
+                    // runs two tiles ahead, so neither wait depends on anything this iteration does
                     if (!bounded_wait(kv_full(vstage), vphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                    if (kstage >= 0 && !bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
                     KSA_TR(0, 40);
                     for (int t = 0; t < nh; ++t) {
                         if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
@@ -266,11 +269,6 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                         KSA_TR(0, 25 + t);
                         if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
                         if (j + 1 < T) {
-                            if (t == 0) {
-                                if (!bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
-                                KSA_TR(0, 41);
-                                tc_fence_after();
-                            }
                             issue_qk(t, kstage);
                             tc_commit(bar(BAR_SFULL + t));
                             KSA_TR(0, 30 + t);
@@ -328,13 +326,6 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { alive = false; break; }
                 sf_phase ^= 1u;
-                if (releaser) {
-                    if (j > 0) release_next();                   // V(j-1)
-                    release_next();                              // K(j)
-                    if (j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
-                } else if ((tid & 127) == 0) {
-                    rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
-                }
                 if (row == 0) KSA_TR(1 + t, 1);
                 tc_fence_after();
                 uint32_t s[128];
@@ -344,6 +335,14 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     uint32_t (&c2)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[64]);
                     uint32_t (&c3)[32] = *reinterpret_cast<uint32_t (*)[32]>(&s[96]);
                     tmem_ld32(tS + 0, c0); tmem_ld32(tS + 32, c1); tmem_ld32(tS + 64, c2); tmem_ld32(tS + 96, c3);
+                }
+                // the stage hand-backs ride on the latency of the loads
+                if (releaser) {
+                    if (j > 0) release_next();                   // V(j-1)
+                    release_next();                              // K(j)
+                    if (j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
+                } else if ((tid & 127) == 0) {
+                    rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
                 }
                 tc_wait_ld();
                 if (row == 0) KSA_TR(1 + t, 2);
