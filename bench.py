@@ -222,7 +222,10 @@ def run_reference(args):
     if rank != 0:
         return 0
     wl, layout = workload_and_layout(args)
-    rows, total = oracle_sample_rows(wl, layout, args.oracle_rows, 1234)
+    # a bounded sample per step, sized so that warm-up plus timed steps stay within a few minutes of host time
+    # (about 9,000 rows in all, at most --oracle-rows per step)
+    per_step = max(32, min(args.oracle_rows, 9000 // max(1, args.warmup + args.steps)))
+    rows, total = oracle_sample_rows(wl, layout, per_step, 1234)
     q, k, v = synth.make_qkv(wl, total)
     times, flops = [], 0.0
     cores = 0
