@@ -45,7 +45,7 @@ cudaError_t launch_bwd_dkv(const BwdArgs& a, cudaStream_t stream);
 // Accumulators -> bf16 dk / dv at the augmented positions.
 cudaError_t launch_bwd_finish(const BwdArgs& a, cudaStream_t stream);
 cudaError_t setup_bwd();
-// dQ and dK / dV of the text rows on the tcgen05 tensor cores (head_dim 128 only).
+// dQ and dK / dV of the text rows on the tcgen05 tensor cores (head_dim 128 and 64).
 cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
 cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
 cudaError_t setup_bwd_tc();
