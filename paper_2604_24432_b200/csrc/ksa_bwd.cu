@@ -527,6 +527,7 @@ cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream)
 cudaError_t launch_bwd_summary(const BwdArgs& a, cudaStream_t stream)
 {
     if (a.m <= 0 || a.max_n_summ <= 0) return cudaSuccess;
+    if (bwd_summary_mma_applies(a)) return launch_bwd_summary_mma(a, stream);
     const int64_t warps = (int64_t)a.max_n_summ * a.Hq;
     dim3 grid((unsigned)((warps + 7) / 8), (unsigned)a.num_seqs, 1);
     if (a.D == 128) ksa_bwd_summary_kernel<128><<<grid, 256, 0, stream>>>(a);

@@ -59,6 +59,12 @@ def _check(name, got, ref):
     ([450], 8, 1, 3, 4, 1, 64, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
     ([1024, 264, 8], 8, 1, 4, 4, 2, 64, 0),           # whole chunks: read in place
     ([1280], 64, 8, 4, 4, 2, 64, 0),
+    # summary-row gradients on mma.sync tiles (8 <= m G <= 128 query rows per chunk and KV head, 12 < k + m <= 128)
+    ([1000, 200], 24, 3, 2, 12, 2, 128, 0),           # 18 rows (a ragged second tile), 27 keys
+    ([600], 56, 8, 1, 4, 4, 64, 0),                   # one query head per KV head, head_dim 64
+    ([1000], 120, 8, 1, 16, 1, 128, 0),               # the largest block: 128 rows, 128 keys
+    ([512, 40], 13, 8, 3, 8, 2, 128, ksa.KSA_FLAG_SUMMARY_TEXT_ONLY),
+    ([4096], 64, 8, 16, 32, 4, 128, 0),               # the 64 + 8 layout with eight query heads per KV head
     # the mma.sync kernels (the on-device cross-check of the tcgen05 kernels)
     ([1000], 8, 1, 16, 8, 2, 128, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
     ([520, 130], 3, 2, 5, 6, 2, 64, ksa.KSA_FLAG_BWD_MMA_SYNC_KERNELS),
