@@ -39,8 +39,8 @@ struct BwdMaps { CUtensorMap qt, dot, kt, vt, ks, vs; };
 cudaError_t launch_bwd_prep(const BwdArgs& a, cudaStream_t stream);
 // Summary query rows: their dQ rows directly, their dK / dV contributions into the accumulators.
 cudaError_t launch_bwd_summary(const BwdArgs& a, cudaStream_t stream);
-// The same for long chunks on mma.sync tiles, one block per (chunk, KV head); launch_bwd_summary dispatches to it when
-// bwd_summary_mma_applies (8 <= m G <= 128 query rows per block, 12 < k + m <= 128 keys per chunk).
+// The same on mma.sync tiles, one block per (chunk, KV head) or per group of short chunks; launch_bwd_summary dispatches
+// to it when bwd_summary_mma_applies (at most 128 query rows m G and 128 keys k + m per chunk).
 bool bwd_summary_mma_applies(const BwdArgs& a);
 cudaError_t launch_bwd_summary_mma(const BwdArgs& a, cudaStream_t stream);
 // Text query rows: dQ (written directly), then dK / dV into the accumulators.

@@ -4,7 +4,8 @@
 // k + m keys (Sec. 2.2.1): with P recomputed from q, k and the forward's lse,
 //   dP = dO V^T,  delta = rowsum(P o dP) (= <dO, O>),  dS = P o (dP - delta),
 //   dQ = scale dS K,  dV = P^T dO,  dK = scale dS^T Q.
-// One block of four warps per (chunk, KV head): Q, dO, K, V rows staged in shared memory (cp.async, 16-byte chunks
+// One block of four warps per (chunk, KV head) -- or per group of consecutive chunks where a chunk alone has fewer than 16
+// query rows: their rows and keys are stacked, and a row sees keys of its own chunk only -- : Q, dO, K, V rows staged in shared memory (cp.async, 16-byte chunks
 // XOR-swizzled by row for ldmatrix).  Phase 1, a warp per 16 query rows: S and dP on the tensor cores, P, delta and
 // dS in registers, dQ = dS K with dS taken from the accumulator registers as the A operand; P and dS also go to shared
 // memory as bf16.  Phase 2, a warp per 16 keys: dV and dK as products over the query rows, with P^T and dS^T read
@@ -12,6 +13,7 @@
 // text keys of the chunk also collect from the text rows' kernels), instead of one per element and query row.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "ksa_bwd.h"
@@ -60,15 +62,17 @@ __device__ __forceinline__ uint32_t bs_sw(uint32_t base, int row, int chunk)
 }
 
 template <int D>
-__global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, int s_pad, int m_pad)
+__global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, int s_pad, int m_pad, int cpb)
 {
     constexpr int CH = D / 8;
     constexpr int KT_MAX = kBsMaxKeys / 16;
     extern __shared__ __align__(128) uint16_t bs_smem[];
     const SeqInfo sq = a.seqs[blockIdx.y];
-    const int j = blockIdx.x, hk = blockIdx.z;
-    if (j >= sq.n_summ / a.m) return;                                  // block-uniform
-    const int G = a.Hq / a.Hkv, tasks = a.m * G, s = a.k + a.m;
+    const int j = blockIdx.x * cpb, hk = blockIdx.z;                   // first chunk of the block
+    const int here = min(cpb, sq.n_summ / a.m - j);                    // chunks of this block
+    if (here <= 0) return;                                             // block-uniform
+    const int G = a.Hq / a.Hkv, per_chunk = a.m * G, s = a.k + a.m;
+    const int tasks = here * per_chunk, keys = here * s;               // stacked query rows and keys
     const int own = (a.flags & 1u) ? 0 : 1;
     const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
     const int pstride = (s_pad + 8) * 2;                               // bytes per row of P / dS (conflict-free for ldmatrix)
@@ -89,15 +93,17 @@ __global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, 
         if (rr < 2 * m_pad) {
             const int t = rr < m_pad ? rr : rr - m_pad;
             if (t < tasks) {
-                const int r = t / G, h = hk * G + (t - r * G);
-                src = rr < m_pad ? a.q + (row0 + a.k + r) * a.q_st + (int64_t)h * a.q_sh + c * 8
-                                 : a.dout + (row0 + a.k + r) * a.do_st + (int64_t)h * a.do_sh + c * 8;
+                const int cc = t / per_chunk, tt = t - cc * per_chunk;
+                const int r = tt / G, h = hk * G + (tt - r * G);
+                const int64_t qrow = row0 + (int64_t)cc * s + a.k + r;
+                src = rr < m_pad ? a.q + qrow * a.q_st + (int64_t)h * a.q_sh + c * 8
+                                 : a.dout + qrow * a.do_st + (int64_t)h * a.do_sh + c * 8;
                 bytes = 16;
             }
             dst = bs_sw<D>(rr < m_pad ? sQ : sG, t, c);
         } else {
             const int kr0 = rr - 2 * m_pad, kr = kr0 < s_pad ? kr0 : kr0 - s_pad;
-            if (kr < s) {
+            if (kr < keys) {
                 src = kr0 < s_pad ? a.kx + (row0 + kr) * a.k_st + (int64_t)hk * a.k_sh + c * 8
                                   : a.v + (row0 + kr) * a.v_st + (int64_t)hk * a.v_sh + c * 8;
                 bytes = 16;
@@ -138,29 +144,33 @@ __global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, 
                 }
             }
         }
-        // rows t0 = 16 mt + g0 and t0 + 8: visible keys [0, nk) (Sec. 2.2.1), lse of the forward pass in log2 units
+        // rows t0 = 16 mt + g0 and t0 + 8: visible keys [lo, lo + nk) of the stacked keys -- the row's own chunk
+        // (Sec. 2.2.1) --, lse of the forward pass in log2 units
         const int t0 = mt * 16 + g0, t1 = t0 + 8;
-        int nk0 = 0, nk1 = 0;
+        int lo0 = 0, lo1 = 0;
+        uint32_t nk0 = 0, nk1 = 0;
         float l0 = 0.f, l1 = 0.f;
         if (t0 < tasks) {
-            const int r = t0 / G, h = hk * G + (t0 - r * G);
-            nk0 = a.k + own * (r + 1);
-            l0 = a.lse[(int64_t)h * a.total_aug + row0 + a.k + r] * 1.4426950408889634f;
+            const int cc = t0 / per_chunk, tt = t0 - cc * per_chunk;
+            const int r = tt / G, h = hk * G + (tt - r * G);
+            lo0 = cc * s; nk0 = (uint32_t)(a.k + own * (r + 1));
+            l0 = a.lse[(int64_t)h * a.total_aug + row0 + (int64_t)cc * s + a.k + r] * 1.4426950408889634f;
         }
         if (t1 < tasks) {
-            const int r = t1 / G, h = hk * G + (t1 - r * G);
-            nk1 = a.k + own * (r + 1);
-            l1 = a.lse[(int64_t)h * a.total_aug + row0 + a.k + r] * 1.4426950408889634f;
+            const int cc = t1 / per_chunk, tt = t1 - cc * per_chunk;
+            const int r = tt / G, h = hk * G + (tt - r * G);
+            lo1 = cc * s; nk1 = (uint32_t)(a.k + own * (r + 1));
+            l1 = a.lse[(int64_t)h * a.total_aug + row0 + (int64_t)cc * s + a.k + r] * 1.4426950408889634f;
         }
         float d0 = 0.f, d1 = 0.f;
 #pragma unroll
         for (int n = 0; n < 2 * KT_MAX; ++n) {
             if (n < 2 * kt_run) {
                 const int key = n * 8 + c2;
-                sc[n][0] = key < nk0 ? bs_ex2(fmaf(sc[n][0], sl2, -l0)) : 0.f;
-                sc[n][1] = key + 1 < nk0 ? bs_ex2(fmaf(sc[n][1], sl2, -l0)) : 0.f;
-                sc[n][2] = key < nk1 ? bs_ex2(fmaf(sc[n][2], sl2, -l1)) : 0.f;
-                sc[n][3] = key + 1 < nk1 ? bs_ex2(fmaf(sc[n][3], sl2, -l1)) : 0.f;
+                sc[n][0] = (uint32_t)(key - lo0) < nk0 ? bs_ex2(fmaf(sc[n][0], sl2, -l0)) : 0.f;
+                sc[n][1] = (uint32_t)(key + 1 - lo0) < nk0 ? bs_ex2(fmaf(sc[n][1], sl2, -l0)) : 0.f;
+                sc[n][2] = (uint32_t)(key - lo1) < nk1 ? bs_ex2(fmaf(sc[n][2], sl2, -l1)) : 0.f;
+                sc[n][3] = (uint32_t)(key + 1 - lo1) < nk1 ? bs_ex2(fmaf(sc[n][3], sl2, -l1)) : 0.f;
                 d0 = fmaf(sc[n][0], dp[n][0], fmaf(sc[n][1], dp[n][1], d0));
                 d1 = fmaf(sc[n][2], dp[n][2], fmaf(sc[n][3], dp[n][3], d1));
             }
@@ -218,10 +228,11 @@ __global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, 
                 const int rl = idx / CH, c = idx - rl * CH;
                 const int t = mt * 16 + rl;
                 if (t >= tasks) continue;
-                const int r = t / G, h = hk * G + (t - r * G);
+                const int cc = t / per_chunk, tt = t - cc * per_chunk;
+                const int r = tt / G, h = hk * G + (tt - r * G);
                 uint4 val;
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(bs_sw<D>(sOw, rl, c)));
-                *reinterpret_cast<uint4*>(a.dq + (row0 + a.k + r) * a.dq_st + (int64_t)h * a.dq_sh + c * 8) = val;
+                *reinterpret_cast<uint4*>(a.dq + (row0 + (int64_t)cc * s + a.k + r) * a.dq_st + (int64_t)h * a.dq_sh + c * 8) = val;
             }
         }
     }
@@ -233,12 +244,13 @@ __global__ void __launch_bounds__(128, 2) ksa_bwd_summary_mma_kernel(BwdArgs a, 
         float* acc_k[2]; float* acc_v[2];
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            const int key = kt * 16 + g0 + 8 * half;
-            if (key < a.k) {
-                const size_t row = (size_t)hk * a.text_rows + sq.text_off + (size_t)j * a.k + key;
+            const int kidx = kt * 16 + g0 + 8 * half;
+            const int kc = kidx / s, key = kidx - kc * s;              // chunk within the block, key within the chunk
+            if (kidx < keys && key < a.k) {
+                const size_t row = (size_t)hk * a.text_rows + sq.text_off + (size_t)(j + kc) * a.k + key;
                 acc_k[half] = a.dkt + row * D; acc_v[half] = a.dvt + row * D;
-            } else if (key < s) {
-                const size_t row = (size_t)hk * a.summ_rows + sq.summ_off + (size_t)j * a.m + (key - a.k);
+            } else if (kidx < keys) {
+                const size_t row = (size_t)hk * a.summ_rows + sq.summ_off + (size_t)(j + kc) * a.m + (key - a.k);
                 acc_k[half] = a.dks + row * D; acc_v[half] = a.dvs + row * D;
             } else {
                 acc_k[half] = nullptr; acc_v[half] = nullptr;
@@ -284,17 +296,26 @@ size_t bs_smem_bytes(int D, int s_pad, int m_pad)
 
 }  // namespace
 
+// Chunks per block: as many as it takes to fill a 16-row tile, within the kernel's row and key limits.
+static int bs_chunks_per_block(const BwdArgs& a)
+{
+    const int G = a.Hq / a.Hkv, per_chunk = a.m * G, s = a.k + a.m;
+    int c = (16 + per_chunk - 1) / per_chunk;
+    c = std::min(c, std::min(kBsMaxKeys / s, kBsMaxRows / per_chunk));
+    return std::max(c, 1);
+}
+
 bool bwd_summary_mma_applies(const BwdArgs& a)
 {
     const int G = a.Hq / a.Hkv;
-    const int s_pad = (a.k + a.m + 15) / 16 * 16, m_pad = (a.m * G + 15) / 16 * 16;
-    return a.m > 0 && s_pad <= kBsMaxKeys && m_pad <= kBsMaxRows && a.m * G >= 8 && a.k + a.m > 12;
+    return a.m > 0 && a.k + a.m <= kBsMaxKeys && a.m * G <= kBsMaxRows;
 }
 
 cudaError_t launch_bwd_summary_mma(const BwdArgs& a, cudaStream_t stream)
 {
     const int G = a.Hq / a.Hkv;
-    const int s_pad = (a.k + a.m + 15) / 16 * 16, m_pad = (a.m * G + 15) / 16 * 16;
+    const int cpb = bs_chunks_per_block(a);
+    const int s_pad = (cpb * (a.k + a.m) + 15) / 16 * 16, m_pad = (cpb * a.m * G + 15) / 16 * 16;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -308,10 +329,11 @@ cudaError_t launch_bwd_summary_mma(const BwdArgs& a, cudaStream_t stream)
             g_bs_done[dev] = true;
         }
     }
-    dim3 grid((unsigned)(a.max_n_summ / a.m), (unsigned)a.num_seqs, (unsigned)a.Hkv);
+    const int max_chunks = a.max_n_summ / a.m;
+    dim3 grid((unsigned)((max_chunks + cpb - 1) / cpb), (unsigned)a.num_seqs, (unsigned)a.Hkv);
     const size_t smem = bs_smem_bytes(a.D, s_pad, m_pad);
-    if (a.D == 128) ksa_bwd_summary_mma_kernel<128><<<grid, 128, smem, stream>>>(a, s_pad, m_pad);
-    else            ksa_bwd_summary_mma_kernel<64><<<grid, 128, smem, stream>>>(a, s_pad, m_pad);
+    if (a.D == 128) ksa_bwd_summary_mma_kernel<128><<<grid, 128, smem, stream>>>(a, s_pad, m_pad, cpb);
+    else            ksa_bwd_summary_mma_kernel<64><<<grid, 128, smem, stream>>>(a, s_pad, m_pad, cpb);
     return cudaGetLastError();
 }
 
