@@ -13,8 +13,9 @@ cudaError_t launch_pack(const KernelArgs& a, cudaStream_t stream);
 
 // Summary rows: each attends to the (at most k + m) keys of its own chunk.
 cudaError_t launch_summary(const KernelArgs& a, cudaStream_t stream);
-// The same for long chunks on mma.sync tiles: one block per (chunk, KV head); launch_summary dispatches to it when
-// summary_mma_applies (m G >= 8 query rows per block, at most 128 of them, at most 128 keys per chunk).
+// The same on mma.sync tiles: one block per (chunk, KV head), or per group of chunks stacked up to 64 query rows;
+// launch_summary dispatches to it for chunks of more than 12 keys when summary_mma_applies (at most 128 query rows m G
+// and 128 keys k + m per chunk).  Chunks of up to 12 keys are faster on the short-chunk kernel (measured).
 bool summary_mma_applies(const KernelArgs& a);
 cudaError_t launch_summary_mma(const KernelArgs& a, int max_chunks, unsigned ny, cudaStream_t stream);
 

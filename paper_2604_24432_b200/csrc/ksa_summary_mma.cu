@@ -3,7 +3,10 @@
 // With many summary tokens per chunk and several query heads per KV head the summary rows of one (chunk, KV head)
 // are a small dense problem: M = m G query rows (summary r of the chunk, query head g of the group), the chunk's
 // k + m keys, head_dim D -- e.g. 64 x 72 x 128 twice over (Q K^T and P V) for the 64 + 8 layout with G = 8.
-// One block of four warps per (chunk, KV head): the chunk's K and V rows and the M query rows are staged in shared
+// Chunks with few query rows are stacked: a block takes an aligned group of consecutive chunks (up to 64 query rows), a
+// row sees the keys of its own chunk only, and chunk j always sits at position j mod group size, so that a row's
+// arithmetic is the same whichever row range a call covers.
+// One block of four warps per (chunk or chunk group, KV head): the K and V rows and the M query rows are staged in shared
 // memory (16-byte chunks XOR-swizzled by row, so that ldmatrix is conflict-free), each warp takes 16-row tiles of the
 // M rows: S = Q K^T over all keys (at most 128, scores stay in registers), the visibility rule of Sec. 2.2.1 -- a
 // summary sees the k text tokens of its chunk and the chunk's summaries up to itself (text only under
@@ -12,6 +15,7 @@
 // tcgen05 tile, and the step is 0.1 - 0.6 % of the forward pass's arithmetic.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "ksa_launch.h"
@@ -61,7 +65,7 @@ __device__ __forceinline__ uint32_t sw_addr(uint32_t base, int row, int chunk)
 }
 
 template <int D>
-__global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, int s_pad, int m_pad)
+__global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, int s_pad, int m_pad, int cpb)
 {
     constexpr int CH = D / 8;                     // 16-byte chunks per row
     constexpr int KT_MAX = kMmaMaxKeys / 16;
@@ -70,12 +74,16 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
     const SeqInfo sq = a.seqs[ranged ? a.r_seq : (int)blockIdx.y];
     const int hk = blockIdx.z;
     const int G = a.Hq / a.Hkv;
-    const int tasks = a.m * G;
+    const int per_chunk = a.m * G, s = a.k + a.m;
     const int j_first = ranged ? a.r_summ0 / a.m : 0;
     const int j_end = ranged ? a.r_summq1 / a.m : sq.n_chunks;
-    const int j = j_first + (int)blockIdx.x;
-    if (j >= j_end) return;                                            // block-uniform
-    const int s = a.k + a.m;
+    // The block takes the chunks of one aligned group [j, j + cpb) that lie in [j_first, j_end): their rows and keys are
+    // stacked, chunk j + cc always at position cc, so that a row's arithmetic does not depend on where a row range starts.
+    const int j = (j_first / cpb + (int)blockIdx.x) * cpb;
+    const int cc_lo = max(0, j_first - j), cc_hi = min(cpb, j_end - j);
+    if (cc_hi <= cc_lo) return;                                        // block-uniform
+    const int tasks = cc_hi * per_chunk, keys = cc_hi * s;             // stacked rows / keys up to the last chunk present
+    const int task_lo = cc_lo * per_chunk, key_lo = cc_lo * s;         // ... from the first chunk present
     const int own = (a.flags & 1u) ? 0 : 1;
     const int64_t row0 = sq.aug_off + (int64_t)j * s;                  // first row of the chunk
     const uint32_t sQ = s_u32(smem);
@@ -88,19 +96,20 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
         const uint16_t* src = a.kx + row0 * a.k_st + (int64_t)hk * a.k_sh;   // a valid address for the zero-filled rows
         uint32_t bytes = 0, dst;
         if (rr < m_pad) {
-            if (rr < tasks) {
-                const int r = rr / G, g = rr - r * G;
-                src = a.q + (row0 + a.k + r) * a.q_st + (int64_t)(hk * G + g) * a.q_sh + c * 8;
+            if (rr >= task_lo && rr < tasks) {
+                const int cc = rr / per_chunk, tt = rr - cc * per_chunk;
+                const int r = tt / G, g = tt - r * G;
+                src = a.q + (row0 + (int64_t)cc * s + a.k + r) * a.q_st + (int64_t)(hk * G + g) * a.q_sh + c * 8;
                 bytes = 16;
             }
             dst = sw_addr<D>(sQ, rr, c);
         } else if (rr < m_pad + s_pad) {
             const int kr = rr - m_pad;
-            if (kr < s) { src = a.kx + (row0 + kr) * a.k_st + (int64_t)hk * a.k_sh + c * 8; bytes = 16; }
+            if (kr >= key_lo && kr < keys) { src = a.kx + (row0 + kr) * a.k_st + (int64_t)hk * a.k_sh + c * 8; bytes = 16; }
             dst = sw_addr<D>(sK, kr, c);
         } else {
             const int vr = rr - m_pad - s_pad;
-            if (vr < s) { src = a.v + (row0 + vr) * a.v_st + (int64_t)hk * a.v_sh + c * 8; bytes = 16; }
+            if (vr >= key_lo && vr < keys) { src = a.v + (row0 + vr) * a.v_st + (int64_t)hk * a.v_sh + c * 8; bytes = 16; }
             dst = sw_addr<D>(sV, vr, c);
         }
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
@@ -115,6 +124,7 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
     const int kt_run = s_pad / 16;
     const float sl2 = a.scale * 1.4426950408889634f;
     for (int mt = warp; mt < m_pad / 16; mt += 4) {
+        if (mt * 16 + 16 <= task_lo || mt * 16 >= tasks) continue;     // no row of this tile is present
         // ---- S = Q K^T: 16 rows x s_pad keys ----
         float sc[2 * KT_MAX][4];
 #pragma unroll
@@ -135,17 +145,24 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
         }
         // ---- visibility (Sec. 2.2.1) and softmax: rows t0 = 16 mt + g0 and t0 + 8 ----
         const int t0 = mt * 16 + g0, t1 = t0 + 8;
-        const int nk0 = a.k + own * (min(t0, tasks - 1) / G + 1);      // visible keys [0, nk) of the row
-        const int nk1 = a.k + own * (min(t1, tasks - 1) / G + 1);
+        // visible keys [lo, lo + nk) of the stacked keys: the row's own chunk (padding rows mimic the last row)
+        int lo0, lo1;
+        uint32_t nk0, nk1;
+        {
+            const int u0 = min(max(t0, task_lo), tasks - 1), u1 = min(max(t1, task_lo), tasks - 1);
+            const int cc0 = u0 / per_chunk, cc1 = u1 / per_chunk;
+            lo0 = cc0 * s; nk0 = (uint32_t)(a.k + own * ((u0 - cc0 * per_chunk) / G + 1));
+            lo1 = cc1 * s; nk1 = (uint32_t)(a.k + own * ((u1 - cc1 * per_chunk) / G + 1));
+        }
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int n = 0; n < 2 * KT_MAX; ++n) {
             if (n < 2 * kt_run) {
                 const int key = n * 8 + c2;
-                sc[n][0] = key < nk0 ? sc[n][0] * sl2 : -INFINITY;
-                sc[n][1] = key + 1 < nk0 ? sc[n][1] * sl2 : -INFINITY;
-                sc[n][2] = key < nk1 ? sc[n][2] * sl2 : -INFINITY;
-                sc[n][3] = key + 1 < nk1 ? sc[n][3] * sl2 : -INFINITY;
+                sc[n][0] = (uint32_t)(key - lo0) < nk0 ? sc[n][0] * sl2 : -INFINITY;
+                sc[n][1] = (uint32_t)(key + 1 - lo0) < nk0 ? sc[n][1] * sl2 : -INFINITY;
+                sc[n][2] = (uint32_t)(key - lo1) < nk1 ? sc[n][2] * sl2 : -INFINITY;
+                sc[n][3] = (uint32_t)(key + 1 - lo1) < nk1 ? sc[n][3] * sl2 : -INFINITY;
                 mx0 = fmaxf(mx0, fmaxf(sc[n][0], sc[n][1]));
                 mx1 = fmaxf(mx1, fmaxf(sc[n][2], sc[n][3]));
             }
@@ -203,9 +220,10 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const int t = half ? t1 : t0;
-                    if (t < tasks) {
-                        const int r = t / G, h = hk * G + (t - r * G);
-                        const int64_t aug = row0 + a.k + r;
+                    if (t >= task_lo && t < tasks) {
+                        const int cc = t / per_chunk, tt = t - cc * per_chunk;
+                        const int r = tt / G, h = hk * G + (tt - r * G);
+                        const int64_t aug = row0 + (int64_t)cc * s + a.k + r;
                         if (ksa_out_row_ok(a, aug, h))
                             a.lse[(int64_t)h * a.total_aug + aug] = ((half ? mx1 : mx0) + log2f(half ? l1 : l0)) * 0.6931471805599453f;
                     }
@@ -217,9 +235,10 @@ __global__ void __launch_bounds__(128, 3) ksa_summary_mma_kernel(KernelArgs a, i
                 const int idx = it * 32 + lane;
                 const int rl = idx / CH, c = idx - rl * CH;
                 const int t = mt * 16 + rl;
-                if (t >= tasks) continue;
-                const int r = t / G, h = hk * G + (t - r * G);
-                const int64_t aug = row0 + a.k + r;
+                if (t < task_lo || t >= tasks) continue;
+                const int cc = t / per_chunk, tt = t - cc * per_chunk;
+                const int r = tt / G, h = hk * G + (tt - r * G);
+                const int64_t aug = row0 + (int64_t)cc * s + a.k + r;
                 if (!ksa_out_row_ok(a, aug, h)) continue;
                 uint4 val;
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(sw_addr<D>(sQ, t, c)));
@@ -234,18 +253,27 @@ bool g_attr_done[64] = {};
 
 }  // namespace
 
+// Chunks per block: short chunks are stacked until the block has up to 64 query rows, within the row and key limits.
+static int summ_chunks_per_block(const KernelArgs& a)
+{
+    const int G = a.Hq / a.Hkv, per_chunk = a.m * G, s = a.k + a.m;
+    int c = 64 / per_chunk;
+    c = std::min(c, std::min(kMmaMaxKeys / s, kMmaMaxRows / per_chunk));
+    return std::max(c, 1);
+}
+
 // True if the kernel takes this shape (rows and keys within its register and shared-memory budget).
 bool summary_mma_applies(const KernelArgs& a)
 {
     const int G = a.Hq / a.Hkv;
-    const int s_pad = (a.k + a.m + 15) / 16 * 16, m_pad = (a.m * G + 15) / 16 * 16;
-    return a.m > 0 && s_pad <= kMmaMaxKeys && m_pad <= kMmaMaxRows && m_pad >= 16 && a.m * G >= 8;
+    return a.m > 0 && a.k + a.m <= kMmaMaxKeys && a.m * G <= kMmaMaxRows;
 }
 
 cudaError_t launch_summary_mma(const KernelArgs& a, int max_chunks, unsigned ny, cudaStream_t stream)
 {
     const int G = a.Hq / a.Hkv;
-    const int s_pad = (a.k + a.m + 15) / 16 * 16, m_pad = (a.m * G + 15) / 16 * 16;
+    const int cpb = summ_chunks_per_block(a);
+    const int s_pad = (cpb * (a.k + a.m) + 15) / 16 * 16, m_pad = (cpb * a.m * G + 15) / 16 * 16;
     const size_t smem = (size_t)(m_pad + 2 * s_pad) * a.D * 2;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -259,9 +287,11 @@ cudaError_t launch_summary_mma(const KernelArgs& a, int max_chunks, unsigned ny,
             g_attr_done[dev] = true;
         }
     }
-    dim3 grid((unsigned)max_chunks, ny, (unsigned)a.Hkv);
-    if (a.D == 128) ksa_summary_mma_kernel<128><<<grid, 128, smem, stream>>>(a, s_pad, m_pad);
-    else            ksa_summary_mma_kernel<64><<<grid, 128, smem, stream>>>(a, s_pad, m_pad);
+    // aligned groups of cpb chunks that the chunk range [j_first, j_first + max_chunks) touches
+    const int j_first = a.r_seq >= 0 ? a.r_summ0 / a.m : 0;
+    dim3 grid((unsigned)((j_first + max_chunks - 1) / cpb - j_first / cpb + 1), ny, (unsigned)a.Hkv);
+    if (a.D == 128) ksa_summary_mma_kernel<128><<<grid, 128, smem, stream>>>(a, s_pad, m_pad, cpb);
+    else            ksa_summary_mma_kernel<64><<<grid, 128, smem, stream>>>(a, s_pad, m_pad, cpb);
     return cudaGetLastError();
 }
 
