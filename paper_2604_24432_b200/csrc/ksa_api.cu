@@ -220,8 +220,9 @@ void build_schedule(const ksa_params* p, HostSchedule& hs, int target_chunks)
 {
     const Eq3 e{p->chunk_len, p->summaries_per_chunk, p->window_chunks};
     const int k = p->chunk_len, m = p->summaries_per_chunk, s = k + m;
-    const int G = p->num_q_heads / p->num_kv_heads;
-    const int heads_per_item = (G % 2 == 0) ? 2 : 1;
+    // two query heads per work item: a pair inside a GQA group shares its K / V tiles; a pair that straddles two KV
+    // heads (multi-head attention, odd group sizes) streams K / V per head; a single head only if the count is odd
+    const int heads_per_item = (p->num_q_heads % 2 == 0) ? 2 : 1;
     struct Tagged { BaseItem it; int32_t chunk; };
     std::vector<Tagged> base;
     hs.chunks.clear();
@@ -294,7 +295,7 @@ static bool schedule_in_range(const ksa_params* p, const HostSchedule& hs)
         const SeqInfo& s = hs.seqs[w.seq];
         if (w.q_tile < 0 || (int64_t)w.q_tile * kTileM >= s.text_pad) return false;
         if (w.n_heads < 1 || w.n_heads > 2 || w.head0 < 0 || w.head0 + w.n_heads > p->num_q_heads) return false;
-        if (w.head0 / G != (w.head0 + w.n_heads - 1) / G) return false;                     // one KV head per item
+        if ((w.head0 + w.n_heads - 1) / G - w.head0 / G > 1) return false;                  // one KV head per item, or one per head
         if (w.ns_tiles < 0 || (int64_t)w.ns_tiles * kTileN > s.summ_pad || w.ns_nomask < 0 || w.ns_nomask > w.ns_tiles) return false;
         if (w.band_lo < 0 || w.band_hi < w.band_lo || w.band_hi != w.q_tile) return false;
         if (w.band_nomask_lo < w.band_lo || w.band_nomask_hi > w.band_hi + 1 || w.band_nomask_hi < w.band_nomask_lo) return false;

@@ -167,7 +167,11 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 if (idx >= a.num_work) break;
                 const WorkItem w = a.work[idx];
                 const SeqInfo sq = a.seqs[w.seq];
+                // the two query heads of an item share a KV head (one K and one V tile per key tile) or, where a pair
+                // straddles two KV heads (multi-head attention, odd group sizes), each has its own: then every key tile
+                // takes four ring stages, K for head 0, K for head 1, V for head 0, V for head 1
                 const int hk = w.head0 / G;
+                const int nsplit = ((w.head0 + w.n_heads - 1) / G != hk) ? 2 : 1;
                 const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
                 if (!bounded_wait(bar(BAR_QEMPTY), q_phase ^ 1u, abort_addr, a.status, kStatusWaitQEmpty)) break;
                 mbar_arrive_expect_tx(bar(BAR_QFULL), (uint32_t)(w.n_heads * Cfg::kTileBytes));
@@ -188,16 +192,17 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     const int zc = sq.chunk0 + (summ ? j * (kTileN / max(a.m, 1)) : (w.band_lo + j - w.ns_tiles) * (kTileN / a.k));
                     const CUtensorMap* mk = summ ? &maps.ks : &maps.kt;
                     const CUtensorMap* mv = summ ? &maps.vs : &maps.vt;
-                    for (int kv = 0; kv < 2; ++kv) {
+                    for (int kvt = 0; kvt < 2 * nsplit && alive; ++kvt) {
+                        const int kv = kvt / nsplit, hkt = hk + kvt % nsplit;
                         if (!bounded_wait(kv_empty(stage), ring_phase ^ 1u, abort_addr, a.status, kStatusWaitKvEmpty)) { alive = false; break; }
                         mbar_arrive_expect_tx(kv_full(stage), (uint32_t)Cfg::kTileBytes);
                         armed_mask |= 1u << stage;
                         armed_parity = (armed_parity & ~(1u << stage)) | (ring_phase << stage);
                         for (int h = 0; h < Cfg::kHalves; ++h)
                             if (a.direct)
-                                tma_load_4d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, 0, zc, hk);
+                                tma_load_4d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, 0, zc, hkt);
                             else
-                                tma_load_3d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, y, hk);
+                                tma_load_3d(sRing + stage * Cfg::kTileBytes + h * 16384, kv ? mv : mk, kv_full(stage), h * 64, y, hkt);
                         if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
                     }
                 }
@@ -240,41 +245,100 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 const WorkItem w = a.work[idx];
                 const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
                 const int nh = w.n_heads;
-                if (!bounded_wait(bar(BAR_QFULL), qf_phase, abort_addr, a.status, kStatusWaitQFull)) break;
-                qf_phase ^= 1u;
-                if (!bounded_wait(kv_full(stage), ring_phase, abort_addr, a.status, kStatusWaitKvFull)) break;
-                tc_fence_after();
-                for (int t = 0; t < nh; ++t) { issue_qk(t, stage); tc_commit(bar(BAR_SFULL + t)); }
-                if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
-                for (int j = 0; j < T && alive; ++j) {
-                    const int vstage = stage; const uint32_t vphase = ring_phase;
+                // one K and one V stage per key tile, or one per query head where the pair straddles two KV heads
+                const int nsplit = ((w.head0 + nh - 1) / G != w.head0 / G) ? 2 : 1;
+                if (nsplit == 1) {
+                // ---- one K and one V stage per key tile (the two heads share a KV head, or a single head) ----
+                    if (!bounded_wait(bar(BAR_QFULL), qf_phase, abort_addr, a.status, kStatusWaitQFull)) break;
+                    qf_phase ^= 1u;
+                    if (!bounded_wait(kv_full(stage), ring_phase, abort_addr, a.status, kStatusWaitKvFull)) break;
+                    tc_fence_after();
+                    for (int t = 0; t < nh; ++t) { issue_qk(t, stage); tc_commit(bar(BAR_SFULL + t)); }
                     if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
-                    int kstage = -1; uint32_t kphase = 0;
-                    if (j + 1 < T) {
-                        kstage = stage; kphase = ring_phase;
+                    for (int j = 0; j < T && alive; ++j) {
+                        const int vstage = stage; const uint32_t vphase = ring_phase;
                         if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
-                    }
-                    KSA_TR(0, 39);
-                    // both stages of this iteration are checked here, while the softmax warps still work on P_0: the ring
-                    // runs two tiles ahead, so neither wait depends on anything this iteration does
-                    if (!bounded_wait(kv_full(vstage), vphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
-                    if (kstage >= 0 && !bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
-                    KSA_TR(0, 40);
-                    for (int t = 0; t < nh; ++t) {
-                        if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
-                        pf_phase[t] ^= 1u;
-                        KSA_TR(0, 20 + t);
-                        tc_fence_after();
-                        issue_pv(t, vstage, j > 0);
-                        KSA_TR(0, 25 + t);
-                        if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
+                        int kstage = -1; uint32_t kphase = 0;
                         if (j + 1 < T) {
-                            issue_qk(t, kstage);
-                            tc_commit(bar(BAR_SFULL + t));
-                            KSA_TR(0, 30 + t);
+                            kstage = stage; kphase = ring_phase;
+                            if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
                         }
+                        KSA_TR(0, 39);
+                        // both stages of this iteration are checked here, while the softmax warps still work on P_0: the ring
+                        // runs two tiles ahead, so neither wait depends on anything this iteration does
+                        if (!bounded_wait(kv_full(vstage), vphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                        if (kstage >= 0 && !bounded_wait(kv_full(kstage), kphase, abort_addr, a.status, kStatusWaitKvFull)) { alive = false; break; }
+                        KSA_TR(0, 40);
+                        for (int t = 0; t < nh; ++t) {
+                            if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
+                            pf_phase[t] ^= 1u;
+                            KSA_TR(0, 20 + t);
+                            tc_fence_after();
+                            issue_pv(t, vstage, j > 0);
+                            KSA_TR(0, 25 + t);
+                            if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
+                            if (j + 1 < T) {
+                                issue_qk(t, kstage);
+                                tc_commit(bar(BAR_SFULL + t));
+                                KSA_TR(0, 30 + t);
+                            }
+                        }
+                        if (!alive) break;
                     }
-                    if (!alive) break;
+                } else {
+                // ---- a pair that straddles two KV heads: every head has its own K and V stage ----
+                    if (!bounded_wait(bar(BAR_QFULL), qf_phase, abort_addr, a.status, kStatusWaitQFull)) break;
+                    qf_phase ^= 1u;
+                    // stage and phase of the K and the V tile of query tile 0 / 1 (scalars: no indexed local arrays)
+                    int kst0, kst1, vst0 = 0, vst1 = 0;
+                    uint32_t kph0, kph1, vph0 = 0, vph1 = 0;
+                    auto take = [&](int& st0, uint32_t& ph0, int& st1, uint32_t& ph1) {   // the next nsplit stages of the ring (not waited for yet)
+                        st0 = stage; ph0 = ring_phase;
+                        if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                        st1 = st0; ph1 = ph0;
+                        if (nsplit == 2) {
+                            st1 = stage; ph1 = ring_phase;
+                            if (++stage == Cfg::kStages) { stage = 0; ring_phase ^= 1u; }
+                        }
+                    };
+                    auto full = [&](int st, uint32_t ph) -> bool { return bounded_wait(kv_full(st), ph, abort_addr, a.status, kStatusWaitKvFull); };
+                    take(kst0, kph0, kst1, kph1);
+                    if (!full(kst0, kph0) || !full(kst1, kph1)) break;
+                    tc_fence_after();
+                    for (int t = 0; t < nh; ++t) { issue_qk(t, t ? kst1 : kst0); tc_commit(bar(BAR_SFULL + t)); }
+                    for (int j = 0; j < T && alive; ++j) {
+                        KSA_TR(0, 39);
+                        take(vst0, vph0, vst1, vph1);
+                        if (j + 1 < T) take(kst0, kph0, kst1, kph1);
+                        // With one K and one V stage per key tile both are checked here, while the softmax warps still work on
+                        // P_0: the ring runs two tiles ahead, so neither wait depends on anything this iteration does.  With
+                        // four stages per key tile the ring runs hardly one tile ahead: each stage is waited for where it is used.
+                        if (nsplit == 1) {
+                            if (!full(vst0, vph0)) { alive = false; break; }
+                            if (j + 1 < T && !full(kst0, kph0)) { alive = false; break; }
+                        }
+                        KSA_TR(0, 40);
+                        for (int t = 0; t < nh; ++t) {
+                            if (!bounded_wait(bar(BAR_PFULL + t), pf_phase[t], abort_addr, a.status, kStatusWaitPFull)) { alive = false; break; }
+                            pf_phase[t] ^= 1u;
+                            KSA_TR(0, 20 + t);
+                            if (nsplit == 2 && !full(t ? vst1 : vst0, t ? vph1 : vph0)) { alive = false; break; }
+                            tc_fence_after();
+                            issue_pv(t, t ? vst1 : vst0, j > 0);
+                            KSA_TR(0, 25 + t);
+                            if (j == T - 1) tc_commit(bar(BAR_OFULL + t));
+                            if (j + 1 < T) {
+                                if (nsplit == 2) {
+                                    if (!full(t ? kst1 : kst0, t ? kph1 : kph0)) { alive = false; break; }
+                                    tc_fence_after();
+                                }
+                                issue_qk(t, t ? kst1 : kst0);
+                                tc_commit(bar(BAR_SFULL + t));
+                                KSA_TR(0, 30 + t);
+                            }
+                        }
+                        if (!alive) break;
+                    }
                 }
             }
             // drain the tensor pipe before TMEM is released
@@ -310,6 +374,7 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             const WorkItem w = a.work[idx];
             if (t >= w.n_heads) { rel_stage = (rel_stage + 2 * (w.ns_tiles + (w.band_hi - w.band_lo + 1))) % Cfg::kStages; continue; }
             const bool releaser = (t == w.n_heads - 1) && (tid & 127) == 0;
+            const int nsplit = ((w.head0 + w.n_heads - 1) / G != w.head0 / G) ? 2 : 1;   // ring stages per K / V tile
             const SeqInfo sq = a.seqs[w.seq];
             const int T = w.ns_tiles + (w.band_hi - w.band_lo + 1);
             const int i_raw = w.q_tile * kTileM + row;
@@ -340,9 +405,10 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                 if (releaser) {
                     if (j > 0) release_next();                   // V(j-1)
                     release_next();                              // K(j)
+                    if (nsplit == 2) { if (j > 0) release_next(); release_next(); }   // ... of the second head
                     if (j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
                 } else if ((tid & 127) == 0) {
-                    rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
+                    rel_stage = (rel_stage + (j > 0 ? 2 : 1) * nsplit) % Cfg::kStages;
                 }
                 tc_wait_ld();
                 if (row == 0) KSA_TR(1 + t, 2);
@@ -434,8 +500,8 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             of_phase ^= 1u;
-            if (releaser) release_next();                        // V(T-1)
-            else if ((tid & 127) == 0) rel_stage = (rel_stage + 1) % Cfg::kStages;
+            if (releaser) { release_next(); if (nsplit == 2) release_next(); }   // V(T-1)
+            else if ((tid & 127) == 0) rel_stage = (rel_stage + nsplit) % Cfg::kStages;
             tc_fence_after();
             const float inv_l = 1.f / l_run;
             const int h = w.head0 + t;
