@@ -252,7 +252,7 @@ int ksa_attn_fwd_host(ksa_ctx* ctx, const void* q_host, const void* k_host, cons
  *     into dense streams (ksa_attn_fwd skips that for whole-chunk batches and then reports
  *     a 256-byte workspace, which is NOT what counts here).  Scratch = 1,280 B + 48 B per
  *     sequence + 48 B per work item (query tiles x pairs of query heads; single heads if
- *     the group size is odd) + the packed streams: 2 * head_dim bytes x
+ *     the number of query heads is odd) + the packed streams: 2 * head_dim bytes x
  *     [(num_q_heads + 2 * num_kv_heads) x text rows + 2 * num_kv_heads x summary rows],
  *     each sequence's rows rounded up to a multiple of 128.  Of the five benchmark
  *     workloads only the 1,024-token one fits.
