@@ -49,7 +49,7 @@ using namespace ptx;
 
 constexpr int kBwdTcThreads = 576;
 constexpr int kBwdTcRegs = 96;                  // 18 warps: five on a scheduler, 5 x 32 x 96 registers fit its file
-constexpr int kBwdSegTiles = 16;                // dK / dV: query tiles (of 128 rows) per CTA
+constexpr int kBwdSegPairs = 64;                // dK / dV: (query tile, query head) pairs per CTA, at least 16 query tiles
 constexpr int kB1Stages = 3, kB2Stages = 2;
 
 // shared memory map (bytes from the 1024-aligned base) for head_dim D
@@ -269,7 +269,7 @@ __device__ __forceinline__ bool bt_stage_free(const BtSmem<D>& sm, int empty0, i
 // =====================================================================================================
 template <int D>
 __global__ void __maxnreg__(kBwdTcRegs)
-ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ)
+ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ, const int seg_tiles)
 {
     extern __shared__ uint8_t bsm_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -294,9 +294,9 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
         qt_lo = (int)(i_min / 128);
         qt_hi = n_qt - 1;
     }
-    const int seg0 = qt_lo + (int)blockIdx.x * kBwdSegTiles;
+    const int seg0 = qt_lo + (int)blockIdx.x * seg_tiles;
     if (seg0 > qt_hi) return;
-    const int seg1 = min(qt_hi + 1, seg0 + kBwdSegTiles);
+    const int seg1 = min(qt_hi + 1, seg0 + seg_tiles);
     const int J = (seg1 - seg0) * G;                                      // streamed tiles: (query tile, query head) pairs
     const int krow0 = (summ ? sq.summ_off : sq.text_off) + kt * 128;      // first row of the key tile in its packed stream
     auto pair_of = [&](int j, int& qt, int& h) { qt = seg0 + j / G; h = hk * G + j % G; };
@@ -851,9 +851,12 @@ cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_
         if (summ && (a.m <= 0 || a.max_n_summ <= 0)) continue;
         const long long span = summ ? n_qt : text_span;
         const int tiles = summ ? (a.max_n_summ + 127) / 128 : n_qt;
-        dim3 grid((unsigned)((span + kBwdSegTiles - 1) / kBwdSegTiles), (unsigned)tiles, (unsigned)(a.num_seqs * a.Hkv));
-        if (a.D == 128) ksa_bwd_dkv_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps, summ);
-        else            ksa_bwd_dkv_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps, summ);
+        // a CTA walks seg query tiles x G heads: 16 tiles with four or more heads per KV head, more with fewer (the
+        // start-up and the final atomics of a CTA are spread over about 64 streamed tiles either way)
+        const int seg = std::max(16, kBwdSegPairs / (a.Hq / a.Hkv));
+        dim3 grid((unsigned)((span + seg - 1) / seg), (unsigned)tiles, (unsigned)(a.num_seqs * a.Hkv));
+        if (a.D == 128) ksa_bwd_dkv_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps, summ, seg);
+        else            ksa_bwd_dkv_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps, summ, seg);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
