@@ -402,13 +402,21 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
                     tmem_ld32(tS + 0, c0); tmem_ld32(tS + 32, c1); tmem_ld32(tS + 64, c2); tmem_ld32(tS + 96, c3);
                 }
                 // the stage hand-backs ride on the latency of the loads
-                if (releaser) {
+                if (nsplit == 2) {
+                    // a stage per head (ring order K_0, K_1, V_0, V_1 per key tile): each query tile's first thread hands
+                    // back its own head's stages as soon as its own scores say they were read; rel_stage stays at the
+                    // item's first stage until the epilogue
+                    if ((tid & 127) == 0) {
+                        if (j > 0) mbar_arrive_relaxed(kv_empty((rel_stage + 4 * (j - 1) + 2 + t) % Cfg::kStages));   // V_t(j-1)
+                        mbar_arrive_relaxed(kv_empty((rel_stage + 4 * j + t) % Cfg::kStages));                         // K_t(j)
+                        if (releaser && j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
+                    }
+                } else if (releaser) {
                     if (j > 0) release_next();                   // V(j-1)
                     release_next();                              // K(j)
-                    if (nsplit == 2) { if (j > 0) release_next(); release_next(); }   // ... of the second head
                     if (j == T - 1) mbar_arrive_relaxed(bar(BAR_QEMPTY));
                 } else if ((tid & 127) == 0) {
-                    rel_stage = (rel_stage + (j > 0 ? 2 : 1) * nsplit) % Cfg::kStages;
+                    rel_stage = (rel_stage + (j > 0 ? 2 : 1)) % Cfg::kStages;
                 }
                 tc_wait_ld();
                 if (row == 0) KSA_TR(1 + t, 2);
@@ -500,8 +508,13 @@ ksa_text_tc_kernel(const __grid_constant__ KernelArgs a, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             of_phase ^= 1u;
-            if (releaser) { release_next(); if (nsplit == 2) release_next(); }   // V(T-1)
-            else if ((tid & 127) == 0) rel_stage = (rel_stage + nsplit) % Cfg::kStages;
+            if (nsplit == 2) {
+                if ((tid & 127) == 0) {
+                    mbar_arrive_relaxed(kv_empty((rel_stage + 4 * (T - 1) + 2 + t) % Cfg::kStages));                   // V_t(T-1)
+                    rel_stage = (rel_stage + 4 * T) % Cfg::kStages;
+                }
+            } else if (releaser) release_next();                 // V(T-1)
+            else if ((tid & 127) == 0) rel_stage = (rel_stage + 1) % Cfg::kStages;
             tc_fence_after();
             const float inv_l = 1.f / l_run;
             const int h = w.head0 + t;
