@@ -95,6 +95,20 @@ def test_edge_shapes(ctx, kernel_flag, lens, k, m, C, Hq, Hkv, D):
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), kernel_flag)
 
 
+@pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
+    ([2048, 1500, 333], 8, 1, 16, 16, 16, 128),   # multi-head attention (the paper's 16/16 model): every pair has two KV heads
+    ([2048, 640], 8, 1, 16, 8, 8, 64),            # the same at head_dim 64, whole chunks (tiles read in place)
+    ([1900], 64, 8, 4, 6, 2, 128),                # three query heads per KV head: pairs (0,1), (2,3) across KV heads, (4,5)
+    ([1500, 700], 8, 1, 5, 10, 2, 128),           # five per KV head
+    ([900], 16, 2, 3, 3, 3, 64),                  # an odd number of query heads: single-head work items
+])
+def test_head_pairs_across_kv_heads(ctx, lens, k, m, C, Hq, Hkv, D):
+    """Work items pair consecutive query heads; where the two belong to different KV heads the kernel streams K and V per
+    head (four ring stages per key tile).  Several tiles, several work items per CTA, packed and in-place inputs."""
+    wl = synth.Workload("mha", 96, lens, Hq, Hkv, D)
+    parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), 0)
+
+
 @pytest.mark.parametrize("strict", [0, STRICT])
 @pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
     ([700, 200], 24, 3, 2, 12, 2, 128),    # 18 query rows per chunk and KV head (two 16-row tiles, one ragged), 27 keys
