@@ -934,10 +934,14 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
     a.dkt = (float*)(ws + bl.dkt); a.dvt = (float*)(ws + bl.dvt); a.dks = (float*)(ws + bl.dks); a.dvs = (float*)(ws + bl.dvs);
     a.status = ctx->d_status;
     a.direct = direct ? 1 : 0;
-    // the four accumulators are contiguous in the workspace: one clear
-    if ((e = cudaMemsetAsync(ws + bl.dkt, 0, bl.total - bl.dkt, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    // The four accumulators are contiguous in the workspace: one clear.  Where one CTA of the tensor-core dK / dV kernel
+    // covers every query tile that sees a text key tile, that launch stores the text keys' rows instead of adding to them:
+    // then only the summary keys' accumulators are cleared and the summary rows' kernel, which adds to both, runs after it.
+    const bool text_stored = !(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS) && bwd_text_keys_stored(a);
+    const size_t clear0 = text_stored ? bl.dks : bl.dkt;
+    if (bl.total > clear0 && (e = cudaMemsetAsync(ws + clear0, 0, bl.total - clear0, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_prep(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if (!text_stored && (e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if (!(p->flags & KSA_FLAG_BWD_MMA_SYNC_KERNELS)) {
         // text rows on the tcgen05 tensor cores, fed by TMA from the packed streams or the caller's tensors
         if (!ctx->bwd_tc_ready) {
@@ -973,6 +977,7 @@ extern "C" __attribute__((visibility("default"))) int ksa_attn_bwd(ksa_ctx* ctx,
         if ((e = launch_bwd_dq(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
         if ((e = launch_bwd_dkv(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     }
+    if (text_stored && (e = launch_bwd_summary(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = launch_bwd_finish(a, stream)) != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += (direct ? 4 : 5) + ((a.m > 0 && a.max_n_summ > 0) ? 2 : 0);
     return KSA_OK;

@@ -52,6 +52,9 @@ cudaError_t setup_bwd();
 // dQ and dK / dV of the text rows on the tcgen05 tensor cores (head_dim 128 and 64).
 cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
 cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream);
+// True if launch_bwd_dkv_tc writes the text keys' accumulator rows with plain stores (one CTA per key tile covers every
+// query tile that sees it): it must then run before anything adds to those rows, and they need no clear.
+bool bwd_text_keys_stored(const BwdArgs& a);
 cudaError_t setup_bwd_tc();
 
 }  // namespace ksa

@@ -269,7 +269,7 @@ __device__ __forceinline__ bool bt_stage_free(const BtSmem<D>& sm, int empty0, i
 // =====================================================================================================
 template <int D>
 __global__ void __maxnreg__(kBwdTcRegs)
-ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ, const int seg_tiles)
+ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__ BwdMaps maps, const int summ, const int seg_tiles, const int store)
 {
     extern __shared__ uint8_t bsm_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -549,11 +549,14 @@ ksa_bwd_dkv_tc_kernel(const __grid_constant__ BwdArgs a, const __grid_constant__
                 tmem_ld32(tacc + c * 32, o);
                 tc_wait_ld();
                 if (key_raw < n_keys) {
+                    // store: this CTA is the only one of its launch for these keys and the first writer of their rows
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        atomicAdd(reinterpret_cast<float4*>(acc + c * 32 + e),
-                                  make_float4(__uint_as_float(o[e]) * mul, __uint_as_float(o[e + 1]) * mul,
-                                              __uint_as_float(o[e + 2]) * mul, __uint_as_float(o[e + 3]) * mul));
+                    for (int e = 0; e < 32; e += 4) {
+                        const float4 val = make_float4(__uint_as_float(o[e]) * mul, __uint_as_float(o[e + 1]) * mul,
+                                                       __uint_as_float(o[e + 2]) * mul, __uint_as_float(o[e + 3]) * mul);
+                        if (store) *reinterpret_cast<float4*>(acc + c * 32 + e) = val;
+                        else atomicAdd(reinterpret_cast<float4*>(acc + c * 32 + e), val);
+                    }
                 }
             }
         }
@@ -843,20 +846,32 @@ cudaError_t launch_bwd_dq_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t
     return cudaGetLastError();
 }
 
+// Query tiles that see a text key tile (an upper bound), and the query tiles a CTA of the dK / dV kernel walks.
+static long long bwd_text_span(const BwdArgs& a)
+{
+    return std::min<long long>(a.max_text_pad / 128, ((long long)a.C + 1) * a.k / 128 + 2);
+}
+static int bwd_seg_tiles(const BwdArgs& a) { return std::max(16, kBwdSegPairs / (a.Hq / a.Hkv)); }
+
+// True if one CTA covers every query tile that sees a text key tile: then the text-key launch writes its rows of the
+// accumulators with plain stores -- it must be their first writer (no clear needed; the summary rows' kernel adds later).
+bool bwd_text_keys_stored(const BwdArgs& a) { return bwd_text_span(a) <= bwd_seg_tiles(a); }
+
 cudaError_t launch_bwd_dkv_tc(const BwdArgs& a, const BwdMaps& maps, cudaStream_t stream)
 {
     const int n_qt = a.max_text_pad / 128;
-    const long long text_span = std::min<long long>(n_qt, ((long long)a.C + 1) * a.k / 128 + 2);
+    const long long text_span = bwd_text_span(a);
     for (int summ = 0; summ < 2; ++summ) {
         if (summ && (a.m <= 0 || a.max_n_summ <= 0)) continue;
         const long long span = summ ? n_qt : text_span;
         const int tiles = summ ? (a.max_n_summ + 127) / 128 : n_qt;
         // a CTA walks seg query tiles x G heads: 16 tiles with four or more heads per KV head, more with fewer (the
         // start-up and the final atomics of a CTA are spread over about 64 streamed tiles either way)
-        const int seg = std::max(16, kBwdSegPairs / (a.Hq / a.Hkv));
+        const int seg = bwd_seg_tiles(a);
+        const int store = (!summ && bwd_text_keys_stored(a)) ? 1 : 0;
         dim3 grid((unsigned)((span + seg - 1) / seg), (unsigned)tiles, (unsigned)(a.num_seqs * a.Hkv));
-        if (a.D == 128) ksa_bwd_dkv_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps, summ, seg);
-        else            ksa_bwd_dkv_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps, summ, seg);
+        if (a.D == 128) ksa_bwd_dkv_tc_kernel<128><<<grid, kBwdTcThreads, BtMap<128>::kSmem, stream>>>(a, maps, summ, seg, store);
+        else            ksa_bwd_dkv_tc_kernel<64><<<grid, kBwdTcThreads, BtMap<64>::kSmem, stream>>>(a, maps, summ, seg, store);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
