@@ -428,7 +428,8 @@ def run_decode(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     ksa_build.build()
-    B, k, C, Hq, Hkv, D = args.decode_batch, 8, 128, 32, 4, 128
+    Hq, Hkv = (int(x) for x in args.decode_heads.split("/"))
+    B, k, C, D = args.decode_batch, 8, 128, 128
     ctx_len = 131072
     steps, warm = args.steps, max(args.warmup, 3)
     spec = ksa.CacheSpec(B, k, C, ctx_len // k + (steps + warm) // k + 2, Hq, Hkv, D, float(np.float32(1.0 / np.sqrt(D))))
@@ -740,6 +741,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode", action="store_true", help="secondary line: the decode path over the Summary KV cache")
     ap.add_argument("--decode-batch", type=int, default=32)
+    ap.add_argument("--decode-heads", default="32/4", help="decode: query heads / KV heads")
     ap.add_argument("--backward", action="store_true", help="secondary line: the backward pass")
     ap.add_argument("--seq-parallel", action="store_true",
                     help="secondary line: one batch shared by all ranks (work-balanced row parts, all-gather of k and v)")
