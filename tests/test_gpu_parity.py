@@ -109,6 +109,14 @@ def test_head_pairs_across_kv_heads(ctx, lens, k, m, C, Hq, Hkv, D):
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), 0)
 
 
+def test_one_million_tokens(ctx):
+    """One sequence of 2^20 text tokens (1,179,648 augmented rows, 8,192 query tiles, up to 1,033 key tiles per work item;
+    8/2 heads keep it at a few GB): sampled rows against the oracle, no bounded wait gave up."""
+    wl = synth.Workload("1m", 7, [1 << 20], 8, 2, 128)
+    parity.check_workload(ctx, wl, synth.LAYOUT_P, 0, n_random=400, seed=3)
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("strict", [0, STRICT])
 @pytest.mark.parametrize("lens,k,m,C,Hq,Hkv,D", [
     ([700, 200], 24, 3, 2, 12, 2, 128),    # 18 query rows per chunk and KV head (two 16-row tiles, one ragged), 27 keys
