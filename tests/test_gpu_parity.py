@@ -109,6 +109,16 @@ def test_head_pairs_across_kv_heads(ctx, lens, k, m, C, Hq, Hkv, D):
     parity.check_workload(ctx, wl, synth.Layout("edge", k, m, C), 0)
 
 
+def test_thousands_of_short_sequences(ctx):
+    """3,000 packed sequences of 1 .. 89 tokens (most shorter than a tile, many shorter than a chunk): sampled rows against
+    the oracle."""
+    rng = np.random.default_rng(5)
+    lens = [int(x) for x in rng.integers(1, 90, size=3000)]
+    wl = synth.Workload("many", 9, lens, 4, 2, 128)
+    parity.check_workload(ctx, wl, synth.Layout("p", 8, 1, 2), 0, n_random=600, seed=4)
+    assert ctx.device_status() == 0
+
+
 def test_one_million_tokens(ctx):
     """One sequence of 2^20 text tokens (1,179,648 augmented rows, 8,192 query tiles, up to 1,033 key tiles per work item;
     8/2 heads keep it at a few GB): sampled rows against the oracle, no bounded wait gave up."""
